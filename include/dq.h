@@ -1,0 +1,168 @@
+/*
+ * dq.h -- C ABI of the format-disaggregated quantized linear layer for NVIDIA
+ * B200 (sm_100a).
+ *
+ * One stored weight matrix W (N x K, out-features x in-features, K contiguous)
+ * is packed once and then served by two phase-specific kernels ("Disaggregated
+ * Quantization", Sec. 2.3 and Fig. 2b): prefill runs a block-scaled NVFP4 x
+ * NVFP4 GEMM on tensor cores after quantising the bf16 activations on the fly,
+ * decode runs a weight-only LUT3 mat-vec against raw bf16 activations.
+ *
+ * Conventions for every entry point
+ *   - returns a dq_status code, never throws, aborts or exits;
+ *   - pointers named *_dev are device pointers on the current CUDA device,
+ *     pointers named *_host are host pointers; the caller owns every buffer;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream); work is
+ *     enqueued on it and the call returns without synchronising;
+ *   - nothing is allocated on the device; scratch comes from the caller;
+ *   - shapes: K % 128 == 0, N % 16 == 0 (else DQ_ERR_SHAPE); row strides in
+ *     elements, multiples of 8; device pointers 16-byte aligned, `packed_dev`
+ *     and `workspace_dev` 1024-byte aligned (else DQ_ERR_ALIGN);
+ *   - NaN/Inf in tensors give unspecified values, never a fault;
+ *   - the device must be compute capability 10.0 (else DQ_ERR_ARCH).
+ */
+#ifndef DQ_H_
+#define DQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dq_weights dq_weights;   /* opaque host-side handle */
+
+enum dq_status {
+    DQ_OK = 0,
+    DQ_ERR_INVALID_ARG = 1,
+    DQ_ERR_SHAPE = 2,
+    DQ_ERR_ALIGN = 3,
+    DQ_ERR_WORKSPACE = 4,
+    DQ_ERR_ARCH = 5,
+    DQ_ERR_CUDA = 6,
+    DQ_ERR_TIMEOUT = 7,
+    DQ_ERR_INTERNAL = 8
+};
+
+/* weight encodings held by a handle (bit mask) */
+enum dq_format {
+    DQ_FMT_NVFP4 = 1,            /* NVFP4 round-to-nearest of the master weights   */
+    DQ_FMT_LUT3 = 2,             /* LUT3 round-to-nearest of the master weights    */
+    DQ_FMT_NVFP4_FROM_LUT3 = 4   /* NVFP4 view re-quantised from the LUT3 codes    */
+};
+
+enum dq_dtype { DQ_DT_BF16 = 0, DQ_DT_FP32 = 1 };
+
+/* Library version (major*10000 + minor*100 + patch). */
+int dq_version(void);
+const char *dq_status_string(int status);
+
+/*
+ * Size of the device buffer dq_pack_weights needs for the requested encodings.
+ * Storage follows App. A.3 "Storage cost": NVFP4 4.5 bit and LUT3 3.5 bit per
+ * weight (codes plus one FP8 scale per 16 weights), plus a 1 KiB header and
+ * padding of the NVFP4 scale tiles to 256 rows.
+ * `formats` must contain at most one of DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3;
+ * DQ_FMT_NVFP4_FROM_LUT3 implies DQ_FMT_LUT3.
+ */
+int dq_packed_bytes(int64_t N, int64_t K, unsigned formats, size_t *bytes_host);
+
+/*
+ * Pack a (fused) weight matrix (App. A.3 "NVFP4-esque two-level scaling",
+ * "NVFP4", "LUT formats"; App. C.2 storage).
+ *   tensor scale  s = max|W| / (6*448) over the whole matrix given (layers an
+ *                 engine fuses are passed concatenated so they share s);
+ *   block scale   d_b = E4M3(extreme_b / (6 s)) per 16 weights along K; for LUT3
+ *                 it carries the sign of the block's maximum-magnitude weight;
+ *   NVFP4 code    nearest E2M1 value of w / (s d_b);
+ *   LUT3 index    nearest level of the 8-entry fp16 codebook, stored bit-planed.
+ *   DQ_FMT_NVFP4_FROM_LUT3 derives the NVFP4 codes from the LUT3 indices
+ *   (Sec. 2.3 autocast) instead of from W.
+ * W_dev: device, row-major, row stride ldw elements, dtype per `w_dtype`.
+ * lut3_codebook_f16_host: 8 fp16 bit patterns, strictly increasing, containing
+ *   0.0 and with maximum 6.0; NULL selects the paper's LUT3A16 grid rounded to fp16.
+ * packed_dev: device buffer of at least dq_packed_bytes bytes; must stay alive
+ *   and unmodified while the handle is used.
+ * *out_host receives a handle owned by the caller (dq_free_weights). The handle
+ * is immutable and may be used from several streams once the pack has finished
+ * on `stream`.
+ */
+int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_t ldw,
+                    unsigned formats, const uint16_t *lut3_codebook_f16_host,
+                    void *packed_dev, size_t packed_bytes, void *stream,
+                    dq_weights **out_host);
+
+/* Frees the host handle only; the packed device buffer belongs to the caller. */
+int dq_free_weights(dq_weights *w);
+
+/* Scratch dq_prefill_linear needs for M tokens (NVFP4 activation codes + scales). */
+int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_host);
+
+/*
+ * Prefill linear (Sec. 1.1 "compute-bound prefill", Sec. 2.3, App. C.1):
+ *   Y[m][n] = bf16( sum_k A^[m][k] * W^[n][k] ),
+ * where A^ is the NVFP4 round-to-nearest of A with the static per-tensor input
+ * scale `act_global_scale` (App. A.3 "NVFP4": s_a in  a^ = s_a * d_b * e2m1) and
+ * W^ the handle's NVFP4 weights; block-scaled FP4 tensor-core GEMM, fp32
+ * accumulation.
+ * A_dev: M x K bf16, row stride lda; Y_dev: M x N bf16, row stride ldy.
+ * act_global_scale must be finite and > 0.  M >= 1.
+ * workspace_dev: at least dq_prefill_workspace_bytes(M) bytes, private to this
+ * call until it has finished on `stream`.
+ */
+int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda,
+                      float act_global_scale, void *Y_dev, int64_t ldy,
+                      void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
+ * Decode linear (Sec. 1.1 "memory-bound decode", App. C.2 "Kernel specification"):
+ *   Y[b][n] = bf16( sum_k X[b][k] * W~[n][k] ),  W~ = s * d_b * codebook[idx],
+ * a weight-only mat-vec / skinny GEMM on the handle's LUT3 weights with raw bf16
+ * activations and fp32 accumulation.  1 <= B <= 64.
+ * X_dev: B x K bf16, row stride ldx; Y_dev: B x N bf16, row stride ldy.
+ */
+int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
+                     void *Y_dev, int64_t ldy, void *stream);
+
+/* ---- parity hooks: canonical encodings, compared bit for bit with the oracle ---- */
+
+/*
+ * Copy one encoding of the handle into canonical layout (all device pointers):
+ *   DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3:
+ *     codes  uint8[N][K/2]  element 2j in the low nibble, 2j+1 in the high nibble,
+ *            code = sign<<3 | index into {0,.5,1,1.5,2,3,4,6} (App. A.3 "NVFP4")
+ *     scales uint8[N][K/16] E4M3
+ *   DQ_FMT_LUT3:
+ *     codes  uint32[N][3][K/32] bit-planes (App. C.2): bit i (LSB = 0) of word j of
+ *            plane p is bit p of the index of weight 32*j + i
+ *     scales uint8[N][K/16] signed E4M3, zero stored as 0x00
+ *   global_scale_dev: one float, the tensor scale s.
+ */
+int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, void *scales_dev,
+                        float *global_scale_dev, void *stream);
+
+/*
+ * The activation quantiser of dq_prefill_linear on its own (App. A.3 "NVFP4",
+ * static input scale), writing canonical layout:
+ *   codes uint8[M][K/2], scales uint8[M][K/16].
+ */
+int dq_quantize_activations(const void *A_dev, int64_t M, int64_t K, int64_t lda,
+                            float act_global_scale, void *codes_dev, void *scales_dev,
+                            void *stream);
+
+/*
+ * Reads the library's device status word for the current device (synchronises
+ * `stream`).  Kernels never trap or spin without bound: a wait that runs out
+ * records DQ_ERR_TIMEOUT and a detail code here and the kernel returns.
+ * The word is cleared by the read.
+ */
+int dq_get_status(void *stream, int *status_host, int *detail_host);
+
+/* Shape queries on a handle. */
+int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsigned *formats_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQ_H_ */

@@ -1,0 +1,206 @@
+"""ctypes binding of include/dq.h.  Argument marshalling only: torch supplies
+device memory and streams, every computation happens inside libdq.so."""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libdq.so"
+
+FMT_NVFP4 = 1
+FMT_LUT3 = 2
+FMT_NVFP4_FROM_LUT3 = 4
+DT_BF16 = 0
+DT_FP32 = 1
+
+# every symbol include/dq.h declares
+SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
+           "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_decode_linear", "dq_export_canonical",
+           "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
+
+
+class DQError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libdq.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                              "(nvcc, sm_100a) first; there is no CPU fallback")
+        L = C.CDLL(str(_LIB_PATH))
+        i64, vp, sz = C.c_int64, C.c_void_p, C.c_size_t
+        L.dq_version.restype = C.c_int
+        L.dq_version.argtypes = []
+        L.dq_status_string.restype = C.c_char_p
+        L.dq_status_string.argtypes = [C.c_int]
+        L.dq_packed_bytes.restype = C.c_int
+        L.dq_packed_bytes.argtypes = [i64, i64, C.c_uint, C.POINTER(sz)]
+        L.dq_pack_weights.restype = C.c_int
+        L.dq_pack_weights.argtypes = [vp, C.c_int, i64, i64, i64, C.c_uint, C.POINTER(C.c_uint16), vp, sz, vp,
+                                      C.POINTER(vp)]
+        L.dq_free_weights.restype = C.c_int
+        L.dq_free_weights.argtypes = [vp]
+        L.dq_prefill_workspace_bytes.restype = C.c_int
+        L.dq_prefill_workspace_bytes.argtypes = [vp, i64, C.POINTER(sz)]
+        L.dq_prefill_linear.restype = C.c_int
+        L.dq_prefill_linear.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp, sz, vp]
+        L.dq_decode_linear.restype = C.c_int
+        L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_export_canonical.restype = C.c_int
+        L.dq_export_canonical.argtypes = [vp, C.c_uint, vp, vp, vp, vp]
+        L.dq_quantize_activations.restype = C.c_int
+        L.dq_quantize_activations.argtypes = [vp, i64, i64, i64, C.c_float, vp, vp, vp]
+        L.dq_get_status.restype = C.c_int
+        L.dq_get_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        L.dq_weights_shape.restype = C.c_int
+        L.dq_weights_shape.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(C.c_uint)]
+        _lib = L
+    return _lib
+
+
+def version() -> int:
+    return int(lib().dq_version())
+
+
+def status_string(code: int) -> str:
+    return lib().dq_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise DQError(code, where)
+
+
+def _stream_ptr(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def packed_bytes(N: int, K: int, formats: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().dq_packed_bytes(N, K, formats, C.byref(out)), "dq_packed_bytes")
+    return int(out.value)
+
+
+class DQWeights:
+    """Handle returned by :func:`pack_weights`; keeps the packed device buffer alive."""
+
+    def __init__(self, handle: int, packed: torch.Tensor, N: int, K: int, formats: int):
+        self.handle = handle
+        self.packed = packed
+        self.N, self.K, self.formats = N, K, formats
+
+    def free(self):
+        if self.handle:
+            lib().dq_free_weights(self.handle)
+            self.handle = 0
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def pack_weights(W: torch.Tensor, formats: int = FMT_NVFP4 | FMT_LUT3, codebook_f16=None, stream=None) -> DQWeights:
+    """dq_pack_weights on a CUDA tensor W (N x K, bf16 or fp32, rows contiguous)."""
+    assert W.is_cuda and W.dim() == 2 and W.stride(1) == 1
+    if W.dtype == torch.bfloat16:
+        dt = DT_BF16
+    elif W.dtype == torch.float32:
+        dt = DT_FP32
+    else:
+        raise TypeError("W must be bf16 or fp32")
+    N, K = W.shape
+    nbytes = packed_bytes(N, K, formats)
+    packed = torch.empty(nbytes + 1024, dtype=torch.uint8, device=W.device)
+    off = (-packed.data_ptr()) % 1024
+    view = packed[off:off + nbytes]
+    cb = None
+    if codebook_f16 is not None:
+        cb = (C.c_uint16 * 8)(*[int(v) for v in codebook_f16])
+    out = C.c_void_p(0)
+    _check(lib().dq_pack_weights(W.data_ptr(), dt, N, K, W.stride(0), formats, cb, view.data_ptr(), nbytes,
+                                 _stream_ptr(stream), C.byref(out)), "dq_pack_weights")
+    if formats & FMT_NVFP4_FROM_LUT3:
+        formats |= FMT_LUT3
+    return DQWeights(out.value, packed, N, K, formats)
+
+
+def prefill_workspace_bytes(w: DQWeights, M: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().dq_prefill_workspace_bytes(w.handle, M, C.byref(out)), "dq_prefill_workspace_bytes")
+    return int(out.value)
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + nbytes]
+
+
+def prefill_linear(w: DQWeights, A: torch.Tensor, act_global_scale: float, out: torch.Tensor = None,
+                   workspace: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """dq_prefill_linear: Y = NVFP4(A) @ NVFP4(W)^T, bf16 out."""
+    assert A.is_cuda and A.dtype == torch.bfloat16 and A.dim() == 2 and A.stride(1) == 1 and A.shape[1] == w.K
+    M = A.shape[0]
+    if out is None:
+        out = torch.empty(M, w.N, dtype=torch.bfloat16, device=A.device)
+    if workspace is None:
+        workspace = alloc_workspace(prefill_workspace_bytes(w, M), A.device)
+    _check(lib().dq_prefill_linear(w.handle, A.data_ptr(), M, A.stride(0), float(act_global_scale), out.data_ptr(),
+                                   out.stride(0), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
+           "dq_prefill_linear")
+    return out
+
+
+def decode_linear(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """dq_decode_linear: Y = X @ LUT3(W)^T, bf16 out, batch 1..64."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    B = X.shape[0]
+    if out is None:
+        out = torch.empty(B, w.N, dtype=torch.bfloat16, device=X.device)
+    _check(lib().dq_decode_linear(w.handle, X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
+                                  _stream_ptr(stream)), "dq_decode_linear")
+    return out
+
+
+def export_canonical(w: DQWeights, fmt: int, stream=None):
+    """Returns (codes, scales, s) in the canonical layouts of include/dq.h (CUDA tensors)."""
+    dev = w.packed.device
+    if fmt in (FMT_NVFP4, FMT_NVFP4_FROM_LUT3):
+        codes = torch.empty(w.N, w.K // 2, dtype=torch.uint8, device=dev)
+    else:
+        codes = torch.empty(w.N, 3, w.K // 32, dtype=torch.int32, device=dev)
+    scales = torch.empty(w.N, w.K // 16, dtype=torch.uint8, device=dev)
+    s = torch.empty(1, dtype=torch.float32, device=dev)
+    _check(lib().dq_export_canonical(w.handle, fmt, codes.data_ptr(), scales.data_ptr(), s.data_ptr(),
+                                     _stream_ptr(stream)), "dq_export_canonical")
+    return codes, scales, s
+
+
+def quantize_activations(A: torch.Tensor, act_global_scale: float, stream=None):
+    assert A.is_cuda and A.dtype == torch.bfloat16 and A.dim() == 2 and A.stride(1) == 1
+    M, K = A.shape
+    codes = torch.empty(M, K // 2, dtype=torch.uint8, device=A.device)
+    scales = torch.empty(M, K // 16, dtype=torch.uint8, device=A.device)
+    _check(lib().dq_quantize_activations(A.data_ptr(), M, K, A.stride(0), float(act_global_scale), codes.data_ptr(),
+                                         scales.data_ptr(), _stream_ptr(stream)), "dq_quantize_activations")
+    return codes, scales
+
+
+def get_status(stream=None):
+    st, det = C.c_int(0), C.c_int(0)
+    _check(lib().dq_get_status(_stream_ptr(stream), C.byref(st), C.byref(det)), "dq_get_status")
+    return int(st.value), int(det.value)

@@ -1,0 +1,327 @@
+// C ABI (include/dq.h): argument checks, handle bookkeeping and kernel launches.
+// No device allocation, no synchronisation except in dq_get_status.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "dq_common.cuh"
+
+namespace dq {
+__device__ StatusWord g_status_word;
+}
+
+struct dq_weights {
+    uint32_t magic;
+    int device;
+    int64_t N, K;
+    unsigned formats;
+    uint8_t *base;
+    dq::PackedLayout layout;
+};
+
+namespace {
+
+constexpr uint32_t kMagic = 0x44515731u;   // "DQW1"
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_arch()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DQ_ERR_CUDA;
+    int major = 0, minor = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return DQ_ERR_CUDA;
+    if (major != 10 || minor != 0) return DQ_ERR_ARCH;
+    return DQ_OK;
+}
+
+int check_shape(int64_t N, int64_t K)
+{
+    if (N <= 0 || K <= 0) return DQ_ERR_SHAPE;
+    if (K % 128 != 0 || N % 16 != 0) return DQ_ERR_SHAPE;
+    if (N > (1ll << 30) || K > (1ll << 30)) return DQ_ERR_SHAPE;
+    return DQ_OK;
+}
+
+int check_formats(unsigned formats)
+{
+    const unsigned all = DQ_FMT_NVFP4 | DQ_FMT_LUT3 | DQ_FMT_NVFP4_FROM_LUT3;
+    if (formats == 0 || (formats & ~all)) return DQ_ERR_INVALID_ARG;
+    if ((formats & DQ_FMT_NVFP4) && (formats & DQ_FMT_NVFP4_FROM_LUT3)) return DQ_ERR_INVALID_ARG;
+    return DQ_OK;
+}
+
+bool valid_handle(const dq_weights *w) { return w != nullptr && w->magic == kMagic; }
+
+dq::StatusWord *status_word_ptr()
+{
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, dq::g_status_word) != cudaSuccess) return nullptr;
+    return reinterpret_cast<dq::StatusWord *>(p);
+}
+
+// default codebook: the paper's LUT3A16 grid (App. A.3 "LUT formats") rounded to fp16
+void default_codebook(uint16_t cb[8])
+{
+    const float grid[8] = {-4.7038f, -2.8698f, -1.3696f, 0.0f, 1.2204f, 2.5285f, 4.0473f, 6.0f};
+    for (int j = 0; j < 8; ++j) cb[j] = __half_as_ushort(__float2half_rn(grid[j]));
+}
+
+bool valid_codebook(const uint16_t cb[8])
+{
+    bool has_zero = false;
+    float prev = 0.0f;
+    for (int j = 0; j < 8; ++j) {
+        const float g = __half2float(__ushort_as_half(cb[j]));
+        if (!std::isfinite(g)) return false;
+        if (j > 0 && !(g > prev)) return false;
+        if (g == 0.0f) { has_zero = true; if (cb[j] != 0) return false; }
+        prev = g;
+    }
+    return has_zero && prev == 6.0f;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dq_version(void) { return 100; }
+
+const char *dq_status_string(int status)
+{
+    switch (status) {
+        case DQ_OK: return "ok";
+        case DQ_ERR_INVALID_ARG: return "invalid argument";
+        case DQ_ERR_SHAPE: return "unsupported shape (need K % 128 == 0, N % 16 == 0)";
+        case DQ_ERR_ALIGN: return "misaligned pointer or stride";
+        case DQ_ERR_WORKSPACE: return "buffer too small";
+        case DQ_ERR_ARCH: return "device is not compute capability 10.0";
+        case DQ_ERR_CUDA: return "CUDA runtime error";
+        case DQ_ERR_TIMEOUT: return "device-side wait ran out";
+        case DQ_ERR_INTERNAL: return "internal error";
+        default: return "unknown status";
+    }
+}
+
+int dq_packed_bytes(int64_t N, int64_t K, unsigned formats, size_t *bytes_host)
+{
+    if (!bytes_host) return DQ_ERR_INVALID_ARG;
+    int st = check_formats(formats);
+    if (st != DQ_OK) return st;
+    st = check_shape(N, K);
+    if (st != DQ_OK) return st;
+    *bytes_host = dq::packed_layout(N, K, formats).total;
+    return DQ_OK;
+}
+
+int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_t ldw, unsigned formats,
+                    const uint16_t *lut3_codebook_f16_host, void *packed_dev, size_t packed_bytes, void *stream,
+                    dq_weights **out_host)
+{
+    if (!W_dev || !packed_dev || !out_host) return DQ_ERR_INVALID_ARG;
+    if (w_dtype != DQ_DT_BF16 && w_dtype != DQ_DT_FP32) return DQ_ERR_INVALID_ARG;
+    int st = check_formats(formats);
+    if (st != DQ_OK) return st;
+    st = check_shape(N, K);
+    if (st != DQ_OK) return st;
+    if (ldw < K || ldw % 8 != 0) return DQ_ERR_ALIGN;
+    if (!aligned(W_dev, 16) || !aligned(packed_dev, 1024)) return DQ_ERR_ALIGN;
+    uint16_t cb[8];
+    if (lut3_codebook_f16_host) std::memcpy(cb, lut3_codebook_f16_host, sizeof(cb));
+    else default_codebook(cb);
+    if (!valid_codebook(cb)) return DQ_ERR_INVALID_ARG;
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    if (formats & DQ_FMT_NVFP4_FROM_LUT3) formats |= DQ_FMT_LUT3;
+    const dq::PackedLayout L = dq::packed_layout(N, K, formats);
+    if (packed_bytes < L.total) return DQ_ERR_WORKSPACE;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint8_t *base = reinterpret_cast<uint8_t *>(packed_dev);
+    dq::PackedHeader *hdr = reinterpret_cast<dq::PackedHeader *>(base);
+    if (cudaMemsetAsync(base, 0, dq::kHeaderBytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_pack_header(hdr, cb, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_absmax(W_dev, w_dtype, N, K, ldw, hdr, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (L.nv_sf_bytes) {
+        if (cudaMemsetAsync(base + L.nv_sf_off, 0, L.nv_sf_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_NVFP4) {
+        if (dq::launch_pack_nvfp4(W_dev, w_dtype, N, K, ldw, hdr, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
+            cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_LUT3) {
+        if (dq::launch_pack_lut3(W_dev, w_dtype, N, K, ldw, hdr,
+                                 reinterpret_cast<uint32_t *>(base + L.lut_planes_off), base + L.lut_sf_off, s) !=
+            cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
+        if (dq::launch_autocast(hdr, reinterpret_cast<const uint32_t *>(base + L.lut_planes_off), base + L.lut_sf_off,
+                                N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
+    dq_weights *w = new (std::nothrow) dq_weights;
+    if (!w) return DQ_ERR_INTERNAL;
+    w->magic = kMagic;
+    cudaGetDevice(&w->device);
+    w->N = N;
+    w->K = K;
+    w->formats = formats;
+    w->base = base;
+    w->layout = L;
+    *out_host = w;
+    return DQ_OK;
+}
+
+int dq_free_weights(dq_weights *w)
+{
+    if (!valid_handle(w)) return DQ_ERR_INVALID_ARG;
+    w->magic = 0;
+    delete w;
+    return DQ_OK;
+}
+
+int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsigned *formats_host)
+{
+    if (!valid_handle(w)) return DQ_ERR_INVALID_ARG;
+    if (N_host) *N_host = w->N;
+    if (K_host) *K_host = w->K;
+    if (formats_host) *formats_host = w->formats;
+    return DQ_OK;
+}
+
+int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_host)
+{
+    if (!valid_handle(w) || !bytes_host || M < 1) return DQ_ERR_INVALID_ARG;
+    const size_t codes = dq::align_up((size_t)M * w->K / 2, 1024);
+    const size_t sf = dq::align_up((size_t)M, dq::kSfAtomRows) * (size_t)(w->K / dq::kBlock);
+    *bytes_host = codes + dq::align_up(sf, 1024);
+    return DQ_OK;
+}
+
+int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda, float act_global_scale,
+                      void *Y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    if (!valid_handle(w) || !A_dev || !Y_dev || !workspace_dev) return DQ_ERR_INVALID_ARG;
+    if (!(w->formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3))) return DQ_ERR_INVALID_ARG;
+    if (M < 1 || M > (1ll << 24)) return DQ_ERR_INVALID_ARG;
+    if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
+    if (lda < w->K || ldy < w->N || lda % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
+    if (!aligned(A_dev, 16) || !aligned(Y_dev, 16) || !aligned(workspace_dev, 1024)) return DQ_ERR_ALIGN;
+    size_t need = 0;
+    dq_prefill_workspace_bytes(w, M, &need);
+    if (workspace_bytes < need) return DQ_ERR_WORKSPACE;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    dq::StatusWord *sw = status_word_ptr();
+    if (!sw) return DQ_ERR_CUDA;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
+    uint8_t *a_codes = ws;
+    uint8_t *a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
+    if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, a_codes, a_sf, 1, s) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    dq::GemmArgs g;
+    g.a_codes = a_codes;
+    g.a_sf = a_sf;
+    g.w_codes = w->base + w->layout.nv_codes_off;
+    g.w_sf = w->base + w->layout.nv_sf_off;
+    g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
+    g.act_scale = act_global_scale;
+    g.Y = Y_dev;
+    g.ldy = ldy;
+    g.M = M;
+    g.N = w->N;
+    g.K = w->K;
+    g.status = sw;
+    if (dq::launch_gemm_nvfp4(g, s) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                     void *stream)
+{
+    if (!valid_handle(w) || !X_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
+    if (!(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
+    if (B < 1 || B > 64) return DQ_ERR_INVALID_ARG;
+    if (ldx < w->K || ldy < w->N || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
+    if (!aligned(X_dev, 16) || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    dq::GemvArgs g;
+    g.planes = reinterpret_cast<const uint32_t *>(w->base + w->layout.lut_planes_off);
+    g.sf = w->base + w->layout.lut_sf_off;
+    g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
+    g.X = X_dev;
+    g.ldx = ldx;
+    g.B = B;
+    g.Y = Y_dev;
+    g.ldy = ldy;
+    g.N = w->N;
+    g.K = w->K;
+    if (dq::launch_gemv_lut3(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, void *scales_dev,
+                        float *global_scale_dev, void *stream)
+{
+    if (!valid_handle(w) || !codes_dev || !scales_dev) return DQ_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const dq::PackedHeader *hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
+    if (format == DQ_FMT_NVFP4 || format == DQ_FMT_NVFP4_FROM_LUT3) {
+        if (!(w->formats & format)) return DQ_ERR_INVALID_ARG;
+        if (dq::launch_export_nvfp4(hdr, w->base + w->layout.nv_codes_off, w->base + w->layout.nv_sf_off, w->N, w->K,
+                                    reinterpret_cast<uint8_t *>(codes_dev), reinterpret_cast<uint8_t *>(scales_dev),
+                                    global_scale_dev, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+        return DQ_OK;
+    }
+    if (format == DQ_FMT_LUT3) {
+        if (!(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
+        if (dq::launch_export_lut3(hdr, reinterpret_cast<const uint32_t *>(w->base + w->layout.lut_planes_off),
+                                   w->base + w->layout.lut_sf_off, w->N, w->K,
+                                   reinterpret_cast<uint32_t *>(codes_dev), reinterpret_cast<uint8_t *>(scales_dev),
+                                   global_scale_dev, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+        return DQ_OK;
+    }
+    return DQ_ERR_INVALID_ARG;
+}
+
+int dq_quantize_activations(const void *A_dev, int64_t M, int64_t K, int64_t lda, float act_global_scale,
+                            void *codes_dev, void *scales_dev, void *stream)
+{
+    if (!A_dev || !codes_dev || !scales_dev) return DQ_ERR_INVALID_ARG;
+    if (M < 1 || K < 1 || K % 128 != 0) return DQ_ERR_SHAPE;
+    if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
+    if (lda < K || lda % 8 != 0 || !aligned(A_dev, 16) || !aligned(codes_dev, 16) || !aligned(scales_dev, 4))
+        return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    if (dq::launch_quant_act(A_dev, M, K, lda, act_global_scale, reinterpret_cast<uint8_t *>(codes_dev),
+                             reinterpret_cast<uint8_t *>(scales_dev), 0,
+                             reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_get_status(void *stream, int *status_host, int *detail_host)
+{
+    if (!status_host) return DQ_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    dq::StatusWord *sw = status_word_ptr();
+    if (!sw) return DQ_ERR_CUDA;
+    dq::StatusWord h;
+    if (cudaMemcpyAsync(&h, sw, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemsetAsync(sw, 0, sizeof(h), s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return DQ_ERR_CUDA;
+    *status_host = h.status;
+    if (detail_host) *detail_host = h.detail;
+    return DQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,392 @@
+// Packers and quantisers: tensor scale, NVFP4 and LUT3 round-to-nearest,
+// LUT3 -> NVFP4 autocast, canonical export, and the activation quantiser of the
+// prefill path.  (App. A.3 "Quantization formats", Sec. 2.3, App. C.2 storage.)
+//
+// Quantiser arithmetic is fp32 with explicit round-to-nearest intrinsics so the
+// compiler cannot contract or reorder it:
+//   rc6 = 1/(6 s);  t = extreme * rc6;  d = E4M3(t);  r = 1/(s * dec(d));  y = x * r
+#include "dq_common.cuh"
+
+namespace dq {
+
+// ---------------------------------------------------------------- converts
+
+__device__ __forceinline__ uint32_t f32_to_e4m3(float t)
+{
+    // cvt packs two values; the second operand lands in the low byte
+    unsigned short out;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(out) : "f"(0.0f), "f"(t));
+    return out & 0xFFu;
+}
+
+__device__ __forceinline__ float e4m3_to_f32(uint32_t b)
+{
+    unsigned short in = (unsigned short)(b & 0xFFu);
+    unsigned int h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(in));
+    return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+
+// two floats -> one byte of E2M1 codes, `lo` in the low nibble
+__device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi)
+{
+    unsigned short out;
+    asm("{\n\t.reg .b8 t;\n\tcvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\tcvt.u16.u8 %0, t;\n\t}"
+        : "=h"(out) : "f"(hi), "f"(lo));
+    return out & 0xFFu;
+}
+
+template <bool FP32IN>
+__device__ __forceinline__ void load16(const void *base, int64_t row, int64_t k0, int64_t ld, float (&x)[16])
+{
+    if (FP32IN) {
+        const float4 *p = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(base) + row * ld + k0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float4 v = __ldg(p + j);
+            x[4 * j] = v.x; x[4 * j + 1] = v.y; x[4 * j + 2] = v.z; x[4 * j + 3] = v.w;
+        }
+    } else {
+        const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(base) + row * ld + k0);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint4 v = __ldg(p + j);
+            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                x[8 * j + 2 * q] = __uint_as_float(w[q] << 16);
+                x[8 * j + 2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+            }
+        }
+    }
+}
+
+// NVFP4 round-to-nearest of one 16-block: returns the E4M3 scale byte, writes 8 code bytes.
+__device__ __forceinline__ uint32_t quant_block_nvfp4(const float (&x)[16], float s, float rc6, uint2 &codes)
+{
+    float a = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(x[i]));
+    const float t = __fmul_rn(a, rc6);
+    const uint32_t d8 = f32_to_e4m3(t);
+    codes = make_uint2(0u, 0u);
+    if ((d8 & 0x7Fu) != 0u) {
+        const float r = __frcp_rn(__fmul_rn(s, e4m3_to_f32(d8)));
+        uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            w0 |= f32x2_to_e2m1x2(__fmul_rn(x[2 * j], r), __fmul_rn(x[2 * j + 1], r)) << (8 * j);
+            w1 |= f32x2_to_e2m1x2(__fmul_rn(x[8 + 2 * j], r), __fmul_rn(x[8 + 2 * j + 1], r)) << (8 * j);
+        }
+        codes = make_uint2(w0, w1);
+    }
+    return d8;
+}
+
+// ------------------------------------------------------------------ header
+
+struct Codebook8 { unsigned short h[8]; };
+
+__global__ void pack_header_kernel(PackedHeader *hdr, Codebook8 cb)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    hdr->amax_bits = 0u;
+    hdr->s = 1.0f;
+    hdr->rc6 = 0.0f;
+    int zero_idx = 0;
+    unsigned int amap = 0;
+    for (int j = 0; j < 8; ++j) {
+        float g = __half2float(__ushort_as_half(cb.h[j]));
+        hdr->lut_levels[j] = g;
+        hdr->lut_f16[j] = cb.h[j];
+        if (g == 0.0f) zero_idx = j;
+        amap |= (f32x2_to_e2m1x2(g, 0.0f) & 0xFu) << (4 * j);
+    }
+    for (int j = 0; j < 7; ++j)
+        hdr->lut_thresholds[j] = __fmul_rn(__fadd_rn(hdr->lut_levels[j], hdr->lut_levels[j + 1]), 0.5f);
+    hdr->lut_thresholds[7] = __int_as_float(0x7f800000);
+    hdr->lut_zero_idx = zero_idx;
+    hdr->autocast_map = amap;
+}
+
+cudaError_t launch_pack_header(PackedHeader *hdr, const uint16_t *codebook_f16_host, cudaStream_t stream)
+{
+    Codebook8 cb;
+    for (int j = 0; j < 8; ++j) cb.h[j] = codebook_f16_host[j];
+    pack_header_kernel<<<1, 32, 0, stream>>>(hdr, cb);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ absmax
+
+template <bool FP32IN>
+__global__ void absmax_kernel(const void *W, int64_t N, int64_t K, int64_t ldw, PackedHeader *hdr)
+{
+    const int64_t nb = K / 16;
+    const int64_t total = N * nb;
+    float a = 0.0f;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        float x[16];
+        load16<FP32IN>(W, i / nb, (i % nb) * 16, ldw, x);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) a = fmaxf(a, fabsf(x[j]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    __shared__ float red[32];
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        a = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.0f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+        if (threadIdx.x == 0) atomicMax(&hdr->amax_bits, __float_as_uint(a));
+    }
+}
+
+__global__ void finalize_scale_kernel(PackedHeader *hdr)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const float amax = __uint_as_float(hdr->amax_bits);
+    const float s = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 2688.0f);      // 6 * 448
+    hdr->s = s;
+    hdr->rc6 = __frcp_rn(__fmul_rn(6.0f, s));
+}
+
+cudaError_t launch_absmax(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw, PackedHeader *hdr,
+                          cudaStream_t stream)
+{
+    const int64_t total = N * (K / 16);
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (w_dtype == DQ_DT_FP32) absmax_kernel<true><<<blocks, 256, 0, stream>>>(W, N, K, ldw, hdr);
+    else absmax_kernel<false><<<blocks, 256, 0, stream>>>(W, N, K, ldw, hdr);
+    finalize_scale_kernel<<<1, 32, 0, stream>>>(hdr);
+    return cudaGetLastError();
+}
+
+// -------------------------------------------------------------- NVFP4 pack
+
+template <bool FP32IN>
+__global__ void pack_nvfp4_kernel(const void *W, int64_t N, int64_t K, int64_t ldw, const PackedHeader *hdr,
+                                  uint8_t *codes, uint8_t *sf)
+{
+    const int64_t nb = K / 16;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * nb) return;
+    const int64_t r = i / nb, b = i % nb;
+    float x[16];
+    load16<FP32IN>(W, r, b * 16, ldw, x);
+    uint2 c;
+    const uint32_t d8 = quant_block_nvfp4(x, hdr->s, hdr->rc6, c);
+    *reinterpret_cast<uint2 *>(codes + r * (K / 2) + b * 8) = c;
+    sf[sf_swizzled_offset(r, b, K)] = (uint8_t)d8;
+}
+
+cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
+                              const PackedHeader *hdr, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream)
+{
+    const int64_t total = N * (K / 16);
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (w_dtype == DQ_DT_FP32) pack_nvfp4_kernel<true><<<blocks, 256, 0, stream>>>(W, N, K, ldw, hdr, codes, sf_swizzled);
+    else pack_nvfp4_kernel<false><<<blocks, 256, 0, stream>>>(W, N, K, ldw, hdr, codes, sf_swizzled);
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------------------- LUT3 pack
+
+// One thread quantises 32 consecutive weights (two 16-blocks) and emits one word of each bit-plane.
+template <bool FP32IN>
+__global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ldw, const PackedHeader *hdr,
+                                 uint32_t *planes, uint8_t *lut_sf)
+{
+    const int64_t nw = K / 32;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * nw) return;
+    const int64_t r = i / nw, j = i % nw;
+    const float s = hdr->s, rc6 = hdr->rc6;
+    float T[7];
+#pragma unroll
+    for (int q = 0; q < 7; ++q) T[q] = hdr->lut_thresholds[q];
+    const int zero_idx = hdr->lut_zero_idx;
+    uint32_t p0 = 0, p1 = 0, p2 = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        float x[16];
+        load16<FP32IN>(W, r, j * 32 + h * 16, ldw, x);
+        // the block's maximum-magnitude weight with its sign; equal magnitudes: the positive one
+        float m = x[0];
+#pragma unroll
+        for (int q = 1; q < 16; ++q) {
+            const float v = x[q];
+            if (fabsf(v) > fabsf(m) || (fabsf(v) == fabsf(m) && v > m)) m = v;
+        }
+        uint32_t d8 = f32_to_e4m3(__fmul_rn(m, rc6));
+        if ((d8 & 0x7Fu) == 0u) d8 = 0u;
+        lut_sf[r * (K / 16) + j * 2 + h] = (uint8_t)d8;
+        const float rr = (d8 != 0u) ? __frcp_rn(__fmul_rn(s, e4m3_to_f32(d8))) : 0.0f;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            int idx = zero_idx;
+            if (d8 != 0u) {
+                const float y = __fmul_rn(x[q], rr);
+                idx = 0;
+#pragma unroll
+                for (int l = 0; l < 7; ++l) idx += (y > T[l]) ? 1 : 0;
+            }
+            const int bit = h * 16 + q;
+            p0 |= (uint32_t)(idx & 1) << bit;
+            p1 |= (uint32_t)((idx >> 1) & 1) << bit;
+            p2 |= (uint32_t)((idx >> 2) & 1) << bit;
+        }
+    }
+    // device layout: [row][K/128 chunks][plane][4 words]
+    uint32_t *dst = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
+    dst[0] = p0; dst[4] = p1; dst[8] = p2;
+}
+
+cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
+                             const PackedHeader *hdr, uint32_t *planes_dev, uint8_t *lut_sf, cudaStream_t stream)
+{
+    const int64_t total = N * (K / 32);
+    const unsigned blocks = (unsigned)((total + 127) / 128);
+    if (w_dtype == DQ_DT_FP32) pack_lut3_kernel<true><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, planes_dev, lut_sf);
+    else pack_lut3_kernel<false><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, planes_dev, lut_sf);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- autocast
+
+// NVFP4 view of the LUT3 codes (Sec. 2.3): level -> nearest E2M1 value, element signs
+// flipped under a negative block scale, block scale |d|, same tensor scale.
+__global__ void autocast_kernel(const PackedHeader *hdr, const uint32_t *planes, const uint8_t *lut_sf, int64_t N,
+                                int64_t K, uint8_t *codes, uint8_t *sf)
+{
+    const int64_t nw = K / 32;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * nw) return;
+    const int64_t r = i / nw, j = i % nw;
+    const uint32_t amap = hdr->autocast_map;
+    const uint32_t *src = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
+    const uint32_t p0 = src[0], p1 = src[4], p2 = src[8];
+    uint32_t out[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t d8 = lut_sf[r * (K / 16) + j * 2 + h];
+        sf[sf_swizzled_offset(r, j * 2 + h, K)] = (uint8_t)(d8 & 0x7Fu);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int bit = h * 16 + q;
+            const uint32_t idx = ((p0 >> bit) & 1u) | (((p1 >> bit) & 1u) << 1) | (((p2 >> bit) & 1u) << 2);
+            uint32_t c = (amap >> (4 * idx)) & 0xFu;
+            if ((d8 & 0x80u) && (c & 0x7u)) c ^= 0x8u;
+            if (d8 == 0u) c = 0u;
+            out[bit / 8] |= c << (4 * (bit % 8));
+        }
+    }
+    *reinterpret_cast<uint4 *>(codes + r * (K / 2) + j * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+cudaError_t launch_autocast(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+                            int64_t K, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream)
+{
+    const int64_t total = N * (K / 32);
+    autocast_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(hdr, planes_dev, lut_sf, N, K, codes,
+                                                                         sf_swizzled);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ export
+
+__global__ void export_nvfp4_kernel(const PackedHeader *hdr, const uint8_t *codes, const uint8_t *sf, int64_t N,
+                                    int64_t K, uint8_t *codes_out, uint8_t *scales_out, float *s_out)
+{
+    const int64_t nb = K / 16;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0 && s_out) *s_out = hdr->s;
+    if (i >= N * nb) return;
+    const int64_t r = i / nb, b = i % nb;
+    *reinterpret_cast<uint2 *>(codes_out + r * (K / 2) + b * 8) =
+        *reinterpret_cast<const uint2 *>(codes + r * (K / 2) + b * 8);
+    scales_out[r * nb + b] = sf[sf_swizzled_offset(r, b, K)];
+}
+
+cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, const uint8_t *sf_swizzled, int64_t N,
+                                int64_t K, uint8_t *codes_out, uint8_t *scales_out, float *s_out,
+                                cudaStream_t stream)
+{
+    const int64_t total = N * (K / 16);
+    export_nvfp4_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, codes, sf_swizzled, N, K,
+                                                                             codes_out, scales_out, s_out);
+    return cudaGetLastError();
+}
+
+__global__ void export_lut3_kernel(const PackedHeader *hdr, const uint32_t *planes, const uint8_t *lut_sf, int64_t N,
+                                   int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out)
+{
+    const int64_t nw = K / 32;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0 && s_out) *s_out = hdr->s;
+    if (i >= N * nw) return;
+    const int64_t r = i / nw, j = i % nw;
+    const uint32_t *src = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
+#pragma unroll
+    for (int p = 0; p < 3; ++p) planes_out[(r * 3 + p) * nw + j] = src[4 * p];
+    scales_out[r * (K / 16) + 2 * j] = lut_sf[r * (K / 16) + 2 * j];
+    scales_out[r * (K / 16) + 2 * j + 1] = lut_sf[r * (K / 16) + 2 * j + 1];
+}
+
+cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+                               int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
+                               cudaStream_t stream)
+{
+    const int64_t total = N * (K / 32);
+    export_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, planes_dev, lut_sf, N, K, planes_out,
+                                                                            scales_out, s_out);
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------- activation quantiser
+
+// bf16 -> NVFP4 with a static tensor scale (App. A.3 "NVFP4").  One thread per
+// 16-block: 32 B in, 8 B of codes out; four neighbouring lanes (one 64-wide k
+// atom) merge their scale bytes into one 32-bit store of the MMA scale layout.
+template <bool SWIZZLED>
+__global__ void __launch_bounds__(256) quant_act_kernel(const __nv_bfloat16 *A, int64_t M, int64_t K, int64_t lda,
+                                                        float s, uint8_t *codes, uint8_t *sf)
+{
+    const int64_t nb = K / 16;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = i < M * nb;
+    const int64_t r = live ? i / nb : 0, b = live ? i % nb : 0;
+    const float rc6 = __frcp_rn(__fmul_rn(6.0f, s));
+    uint32_t d8 = 0;
+    if (live) {
+        float x[16];
+        load16<false>(A, r, b * 16, lda, x);
+        uint2 c;
+        d8 = quant_block_nvfp4(x, s, rc6, c);
+        *reinterpret_cast<uint2 *>(codes + r * (K / 2) + b * 8) = c;
+    }
+    // K % 64 == 0, so lanes 4q..4q+3 always hold the four blocks of one k atom of one row
+    uint32_t w = d8 << (8 * (threadIdx.x & 3));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    w |= __shfl_xor_sync(0xffffffffu, w, 2);
+    if (live && (threadIdx.x & 3) == 0) {
+        if (SWIZZLED) *reinterpret_cast<uint32_t *>(sf + sf_swizzled_offset(r, b, K)) = w;
+        else *reinterpret_cast<uint32_t *>(sf + r * nb + b) = w;
+    }
+}
+
+cudaError_t launch_quant_act(const void *A_bf16, int64_t M, int64_t K, int64_t lda, float act_scale, uint8_t *codes,
+                             uint8_t *sf, int swizzled, cudaStream_t stream)
+{
+    const int64_t total = M * (K / 16);
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const __nv_bfloat16 *A = reinterpret_cast<const __nv_bfloat16 *>(A_bf16);
+    if (swizzled) quant_act_kernel<true><<<blocks, 256, 0, stream>>>(A, M, K, lda, act_scale, codes, sf);
+    else quant_act_kernel<false><<<blocks, 256, 0, stream>>>(A, M, K, lda, act_scale, codes, sf);
+    return cudaGetLastError();
+}
+
+}  // namespace dq

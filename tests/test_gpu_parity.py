@@ -1,0 +1,266 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Codes and scales bit for bit; GEMM / GEMV outputs
+within relative Frobenius error 2e-3 and, per element, one bf16 ulp plus
+1e-4 * sum_k |a*w| (see parity_utils)."""
+import numpy as np
+import pytest
+import torch
+
+import dq_inputs
+from parity_utils import check_outputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dq():
+    import __graft_entry__ as g
+    g.build()
+    import paper_2609_26333_b200 as dq
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    assert torch.cuda.get_device_capability(0) == (10, 0), "this library targets sm_100a only"
+    return dq
+
+
+DEV = "cuda:0"
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def _status_ok(dq):
+    torch.cuda.synchronize()
+    st, det = dq.get_status()
+    assert st == 0, f"device status {dq.status_string(st)} detail {det}"
+
+
+_ref_cache = {}
+
+
+def _layer(oracle, N, K, seed, std=0.02, dtype=torch.bfloat16):
+    key = (N, K, seed, std, dtype)
+    if key not in _ref_cache:
+        if dtype == torch.bfloat16:
+            W = dq_inputs.gaussian_bf16(N, K, std, seed)
+            Wf = dq_inputs.bf16_to_f32_numpy(W)
+        else:
+            g = torch.Generator().manual_seed(seed)
+            W = torch.randn(N, K, generator=g, dtype=torch.float32) * std
+            Wf = W.numpy()
+        _ref_cache[key] = (W, oracle.pack_weights(Wf))
+    return _ref_cache[key]
+
+
+# shapes: tiny config; ragged multi-tile (N not a multiple of the tile, K with a 128 tail); several tiles
+PACK_SHAPES = [(512, 256, 0), (144, 384, 31), (784, 1152, 32)]
+
+
+@pytest.mark.parametrize("N,K,seed", PACK_SHAPES)
+def test_pack_bit_exact(dq, oracle, N, K, seed):
+    W, ref = _layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV))
+    codes, scales, s = dq.export_canonical(w, dq.FMT_NVFP4)
+    planes, lsc, s2 = dq.export_canonical(w, dq.FMT_LUT3)
+    _status_ok(dq)
+    assert np.float32(_np(s)[0]) == np.float32(ref["s"]) and _np(s2)[0] == _np(s)[0]
+    assert np.array_equal(_np(scales), ref["nvfp4_scales"])
+    assert np.array_equal(_np(codes), ref["nvfp4_codes"])
+    assert np.array_equal(_np(lsc), ref["lut3_scales"])
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"])
+
+
+def test_pack_fp32_master_and_strided_rows(dq, oracle):
+    N, K = 160, 256
+    W, ref = _layer(oracle, N, K, 33, dtype=torch.float32)
+    big = torch.zeros(N, K + 64, dtype=torch.float32, device=DEV)
+    big[:, :K] = W.to(DEV)
+    w = dq.pack_weights(big[:, :K])
+    codes, scales, s = dq.export_canonical(w, dq.FMT_NVFP4)
+    planes, lsc, _ = dq.export_canonical(w, dq.FMT_LUT3)
+    _status_ok(dq)
+    assert np.array_equal(_np(codes), ref["nvfp4_codes"]) and np.array_equal(_np(scales), ref["nvfp4_scales"])
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"]) and np.array_equal(_np(lsc), ref["lut3_scales"])
+
+
+def test_pack_degenerate_tensors(dq, oracle):
+    N, K = 32, 128
+    # all zero: s = 1, zero scales, zero codes, LUT index of the 0.0 level
+    Z = torch.zeros(N, K, dtype=torch.bfloat16)
+    ref = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(Z))
+    w = dq.pack_weights(Z.to(DEV))
+    codes, scales, s = dq.export_canonical(w, dq.FMT_NVFP4)
+    planes, lsc, _ = dq.export_canonical(w, dq.FMT_LUT3)
+    assert _np(s)[0] == 1.0 and not _np(codes).any() and not _np(scales).any() and not _np(lsc).any()
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"])
+    # sign ties, zero blocks, a single huge outlier (block-scale underflow elsewhere)
+    X = dq_inputs.gaussian_bf16(N, K, 0.02, 34)
+    X[0, :16] = 0
+    X[1, 0], X[1, 5] = 0.5, -0.5
+    X[2, 3], X[2, 9] = -0.75, 0.75
+    X[3, 7] = 3.0e4
+    ref = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(X))
+    w = dq.pack_weights(X.to(DEV))
+    codes, scales, s = dq.export_canonical(w, dq.FMT_NVFP4)
+    planes, lsc, _ = dq.export_canonical(w, dq.FMT_LUT3)
+    _status_ok(dq)
+    assert np.float32(_np(s)[0]) == np.float32(ref["s"])
+    assert np.array_equal(_np(codes), ref["nvfp4_codes"]) and np.array_equal(_np(scales), ref["nvfp4_scales"])
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"]) and np.array_equal(_np(lsc), ref["lut3_scales"])
+
+
+def test_autocast_view_bit_exact(dq, oracle):
+    N, K = 272, 512
+    W, ref = _layer(oracle, N, K, 35)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4_FROM_LUT3)
+    codes, scales, s = dq.export_canonical(w, dq.FMT_NVFP4_FROM_LUT3)
+    planes, lsc, _ = dq.export_canonical(w, dq.FMT_LUT3)
+    _status_ok(dq)
+    ac, asc = oracle.autocast_lut3_to_nvfp4(ref["lut3_planes"], ref["lut3_scales"])
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"])
+    assert np.array_equal(_np(codes), ac) and np.array_equal(_np(scales), asc)
+
+
+def test_custom_codebook(dq, oracle):
+    N, K = 64, 256
+    W, _ = _layer(oracle, N, K, 36)
+    cb = np.array([oracle.f16_encode(v) for v in (-5, -3, -1.5, 0, 1, 2.25, 4, 6)], dtype=np.uint16)
+    Wf = dq_inputs.bf16_to_f32_numpy(W)
+    ref = oracle.pack_weights(Wf, cb)
+    w = dq.pack_weights(W.to(DEV), codebook_f16=cb)
+    planes, lsc, _ = dq.export_canonical(w, dq.FMT_LUT3)
+    assert np.array_equal(_np(planes).view(np.uint32), ref["lut3_planes"]) and np.array_equal(_np(lsc), ref["lut3_scales"])
+    X = dq_inputs.gaussian_bf16(2, K, 1.0, 37)
+    Y = dq.decode_linear(w, X.to(DEV))
+    _status_ok(dq)
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X), ref["lut3_planes"], ref["lut3_scales"], ref["s"], cb)
+    check_outputs(_f64(Y), Yr, S, "custom codebook decode")
+
+
+@pytest.mark.parametrize("M,K,kind", [(64, 256, "gauss"), (300, 640, "gauss"), (257, 1024, "student")])
+def test_activation_quantiser_bit_exact(dq, oracle, M, K, kind):
+    if kind == "gauss":
+        A = dq_inputs.gaussian_bf16(M, K, 1.0, 40 + M)
+    else:
+        A = dq_inputs.student_t_outlier_bf16(M, K, 41)
+    sa = dq_inputs.static_act_scale(A)
+    codes, scales = dq.quantize_activations(A.to(DEV), sa)
+    _status_ok(dq)
+    rc, rs = oracle.quant_nvfp4(dq_inputs.bf16_to_f32_numpy(A), sa)
+    assert np.array_equal(_np(scales), rs)
+    assert np.array_equal(_np(codes), rc)
+    # a static scale that is too small saturates instead of misbehaving
+    codes2, scales2 = dq.quantize_activations(A.to(DEV), sa / 64)
+    rc2, rs2 = oracle.quant_nvfp4(dq_inputs.bf16_to_f32_numpy(A), sa / 64)
+    assert np.array_equal(_np(scales2), rs2) and np.array_equal(_np(codes2), rc2)
+    assert (rs2 == 0x7E).any()
+
+
+PREFILL_SHAPES = [
+    # M, N, K, seed : tiny config (M below one tile); ragged tiles with a K tail; several tiles per CTA
+    (64, 512, 256, 0),
+    (300, 784, 640, 51),
+    (1, 256, 128, 52),
+    (129, 272, 1152, 53),
+    (640, 1536, 2048, 54),
+]
+
+
+@pytest.mark.parametrize("M,N,K,seed", PREFILL_SHAPES)
+def test_prefill_parity(dq, oracle, M, N, K, seed):
+    W, ref = _layer(oracle, N, K, seed)
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, seed + 7)
+    sa = dq_inputs.static_act_scale(A)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    Y = dq.prefill_linear(w, A.to(DEV), sa)
+    _status_ok(dq)
+    Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa, ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, f"prefill {M}x{N}x{K}")
+    # repeated call on the same handle and workspace gives the same bits
+    Y2 = dq.prefill_linear(w, A.to(DEV), sa)
+    assert torch.equal(Y, Y2)
+
+
+def test_prefill_strided_output_and_autocast_weights(dq, oracle):
+    M, N, K = 200, 528, 384
+    W, ref = _layer(oracle, N, K, 55)
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, 56)
+    sa = dq_inputs.static_act_scale(A)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4_FROM_LUT3)
+    out = torch.full((M, N + 16), 7.0, dtype=torch.bfloat16, device=DEV)
+    dq.prefill_linear(w, A.to(DEV), sa, out=out[:, :N])
+    _status_ok(dq)
+    assert torch.all(out[:, N:] == 7.0)
+    ac, asc = oracle.autocast_lut3_to_nvfp4(ref["lut3_planes"], ref["lut3_scales"])
+    Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa, ac, asc, ref["s"])
+    check_outputs(_f64(out[:, :N]), Yr, S, "prefill on autocast weights")
+
+
+def test_prefill_outlier_activations(dq, oracle):
+    M, N, K = 256, 512, 1024
+    W, ref = _layer(oracle, N, K, 57)
+    A = dq_inputs.student_t_outlier_bf16(M, K, 58)
+    sa = dq_inputs.static_act_scale(A)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    Y = dq.prefill_linear(w, A.to(DEV), sa)
+    _status_ok(dq)
+    Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa, ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, "prefill with heavy-tailed activations")
+
+
+DECODE_SHAPES = [(512, 256, 0), (144, 384, 61), (784, 1152, 62), (2048, 4096, 63)]
+
+
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES)
+@pytest.mark.parametrize("B", [1, 2, 3, 8, 17, 64])
+def test_decode_parity(dq, oracle, N, K, seed, B):
+    W, ref = _layer(oracle, N, K, seed)
+    X = dq_inputs.gaussian_bf16(B, K, 1.0, seed + 100 + B)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    Y = dq.decode_linear(w, X.to(DEV))
+    _status_ok(dq)
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, f"decode {B}x{N}x{K}")
+
+
+def test_decode_one_hot_and_strided(dq, oracle):
+    N, K = 256, 512
+    W, ref = _layer(oracle, N, K, 64)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    What = oracle.dequant_lut3(ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    X = torch.zeros(4, K + 8, dtype=torch.bfloat16)
+    ks = [0, 17, 130, 511]
+    for b, k in enumerate(ks):
+        X[b, k] = 1.0
+    out = torch.full((4, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+    dq.decode_linear(w, X.to(DEV)[:, :K], out=out[:, :N])
+    _status_ok(dq)
+    assert torch.all(out[:, N:] == -3.0)
+    got = _f64(out[:, :N])
+    for b, k in enumerate(ks):      # one dequantised column, rounded to bf16
+        want = torch.from_numpy(What[:, k]).to(torch.bfloat16).float().numpy().astype(np.float64)
+        assert np.array_equal(got[b], want)
+
+
+def test_calls_reject_wrong_handle_use(dq, oracle):
+    N, K = 64, 128
+    W, _ = _layer(oracle, N, K, 65)
+    w_lut = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    w_nv = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    A = dq_inputs.gaussian_bf16(4, K, 1.0, 66).to(DEV)
+    with pytest.raises(dq.DQError) as e:
+        dq.prefill_linear(w_lut, A, 1.0)
+    assert e.value.code == 1
+    with pytest.raises(dq.DQError) as e:
+        dq.decode_linear(w_nv, A)
+    assert e.value.code == 1
+    with pytest.raises(dq.DQError) as e:
+        dq.prefill_linear(w_nv, A, 1.0, workspace=torch.empty(1024, dtype=torch.uint8, device=DEV)[:16])
+    assert e.value.code in (3, 4)
+    with pytest.raises(dq.DQError):
+        dq.prefill_linear(w_nv, A, -1.0)
+    _status_ok(dq)
