@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the format-disaggregated quantized linear layer on B200.
+
+One step = one pass of the serving hot path over one batch of synthetic input on
+one packed layer: dq_prefill_quantize + dq_prefill_gemm (NVFP4 prefill linear for
+M tokens) followed by dq_decode_linear (LUT3 decode, batch 1).  Packing is a
+load-time operation; it is timed once and reported as `pack_ms`.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an
+independent replica of the same workload; there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np
+import torch
+
+import dq_inputs
+
+METRIC = "NVFP4 prefill GEMM TFLOP/s & LUT3 decode GEMV GB/s, % of B200 roofline"
+DEFAULT_WORKLOAD = "c3_gate_up27b"
+L2_BYTES = 126 * 1024 * 1024
+
+# DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum);
+# see profiles/ for the captures these come from.  None = not captured for that workload.
+NCU_TRAFFIC_BYTES = {
+    ("gemm", "c3_gate_up27b"): None,
+    ("gemv", "c3_gate_up27b"): None,
+}
+
+
+def load_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_burst": float(d["bf16_tflops"]),
+                "bf16_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.05):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        self.h = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            props = torch.cuda.get_device_properties(device_index)
+            h = None
+            uuid = getattr(props, "uuid", None)
+            if uuid is not None:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+                except Exception:
+                    h = None
+            if h is None:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                phys = int(vis.split(",")[device_index]) if vis and vis.split(",")[device_index].isdigit() else device_index
+                h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.h = h
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.h = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_sample_run(cfg, W_f32, ref, A_f32, sa, X_f32, rows):
+    """One bounded pass of the oracle: `rows` prefill tokens + one decode token."""
+    import oracle
+    t0 = time.perf_counter()
+    oracle.prefill_linear(A_f32[:rows], sa, ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    t1 = time.perf_counter()
+    oracle.decode_linear(X_f32, ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    rows = args.ref_rows
+    W = dq_inputs.make_weight(cfg)
+    W_f32 = dq_inputs.bf16_to_f32_numpy(W)
+    A = dq_inputs.make_activations(cfg, rows)
+    sa = dq_inputs.static_act_scale(A)
+    A_f32 = dq_inputs.bf16_to_f32_numpy(A)
+    X_f32 = dq_inputs.bf16_to_f32_numpy(dq_inputs.make_activations(cfg, 1, salt=2))
+    ref = oracle.pack_weights(W_f32)
+    for _ in range(args.warmup):
+        oracle_sample_run(cfg, W_f32, ref, A_f32, sa, X_f32, rows)
+    tp = td = 0.0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        a, b = oracle_sample_run(cfg, W_f32, ref, A_f32, sa, X_f32, rows)
+        tp += a
+        td += b
+    total = time.perf_counter() - t0
+    tflops = 2.0 * rows * cfg.N * cfg.K * args.steps / tp / 1e12
+    dec_bytes = 0.4375 * cfg.N * cfg.K + 2 * cfg.K + 2 * cfg.N + 4
+    sample = f"{rows} of {cfg.M} prefill rows (dequantise + fp64 matmul of the whole N x K layer) + 1 decode token per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "N": cfg.N, "K": cfg.K, "M": cfg.M, "decode_batch": 1, "sample": sample},
+        "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "decode": {"value": dec_bytes * args.steps / td / 1e9, "unit": "GB/s"},
+        "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(dq_inputs.CONFIGS))
+    ap.add_argument("--mnk", default=None, help="M,N,K of an ad-hoc Gaussian layer (profiling small cases)")
+    ap.add_argument("--impl", default="dq", choices=["dq", "reference"])
+    ap.add_argument("--decode-batch", type=int, default=1)
+    ap.add_argument("--copies", type=int, default=0, help="rotating packed-weight copies (0 = enough to exceed 2x L2)")
+    ap.add_argument("--ref-rows", type=int, default=128, help="prefill rows per oracle step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "dq" else args.warmup
+    cfg = dq_inputs.CONFIGS[args.workload]
+    if args.mnk:
+        m, n, k = (int(v) for v in args.mnk.split(","))
+        cfg = dq_inputs.LayerConfig(f"adhoc_{m}x{n}x{k}", N=n, K=k, M=m, cfg_id=9)
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    import __graft_entry__ as g
+    if rank == 0:
+        g.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2609_26333_b200 as dq
+    dq.lib()
+
+    peaks = load_peaks()
+    M, N, K, B = cfg.M, cfg.N, cfg.K, args.decode_batch
+
+    # ---- inputs (seeded, CPU-drawn, same bytes the oracle would see) ----
+    W = dq_inputs.make_weight(cfg).to(dev)
+    A_host = dq_inputs.make_activations(cfg, M).pin_memory()
+    X_host = dq_inputs.make_activations(cfg, B, salt=2).pin_memory()
+    sa = dq_inputs.static_act_scale(A_host)
+    A = A_host.to(dev)
+    X = X_host.to(dev)
+
+    packed_bytes = dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3)
+    copies = args.copies or max(2, int(np.ceil(2.5 * L2_BYTES / (0.4375 * N * K))))
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ws = []
+    for c in range(copies):
+        if c == 1:
+            e0.record()
+        ws.append(dq.pack_weights(W))
+        if c == 1:
+            e1.record()
+    torch.cuda.synchronize()
+    pack_ms = e0.elapsed_time(e1) if copies > 1 else None
+    del W
+
+    workspace = dq.alloc_workspace(dq.prefill_workspace_bytes(ws[0], M), dev)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    Yd = torch.empty(B, N, dtype=torch.bfloat16, device=dev)
+
+    def step(i, ev=None):
+        w = ws[i % copies]
+        if ev is not None:
+            ev[0].record()
+        dq.prefill_quantize(w, A, sa, workspace)
+        if ev is not None:
+            ev[1].record()
+        dq.prefill_gemm(w, M, sa, Y, workspace)
+        if ev is not None:
+            ev[2].record()
+        dq.decode_linear(w, X, out=Yd)
+        if ev is not None:
+            ev[3].record()
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    st, det = dq.get_status()
+    if st != 0:
+        raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after warm-up")
+
+    # ---- timed region: exactly K steps ----
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_start.record()
+    for i in range(args.steps):
+        step(args.warmup + i, evs[i])
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    q_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    g_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    d_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    st, det = dq.get_status()
+    if st != 0:
+        raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the timed region")
+
+    # ---- end to end: pinned host buffers, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        Y_host = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+        Yd_host = torch.empty(B, N, dtype=torch.bfloat16).pin_memory()
+        A2, X2 = torch.empty_like(A), torch.empty_like(X)
+
+        def e2e_step(i, ev=None):
+            w = ws[i % copies]
+            if ev is not None:
+                ev[0].record()
+            A2.copy_(A_host, non_blocking=True)
+            dq.prefill_linear(w, A2, sa, out=Y, workspace=workspace)
+            Y_host.copy_(Y, non_blocking=True)
+            if ev is not None:
+                ev[1].record()
+            X2.copy_(X_host, non_blocking=True)
+            dq.decode_linear(w, X2, out=Yd)
+            Yd_host.copy_(Yd, non_blocking=True)
+            if ev is not None:
+                ev[2].record()
+
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        n_e2e = max(3, min(args.steps, 10))
+        ee = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_e2e)]
+        for i in range(n_e2e):
+            e2e_step(i, ee[i])
+        torch.cuda.synchronize()
+        p_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ee]))
+        dd_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ee]))
+        e2e = {"prefill_ms": p_ms, "decode_ms": dd_ms, "steps": n_e2e}
+
+    # ---- max over ranks ----
+    times = torch.tensor([total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0,
+                          e2e["decode_ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms = [float(v) for v in times.cpu()]
+
+    flops = 2.0 * M * N * K
+    dec_bytes = 0.4375 * N * K + 2.0 * B * K + 2.0 * B * N + 4
+    quant_bytes = 2.5625 * M * K
+    prefill_tflops = world * flops / ((q_ms + g_ms) * 1e-3) / 1e12
+    gemm_tflops = flops / (g_ms * 1e-3) / 1e12
+    decode_gbs = dec_bytes / (d_ms * 1e-3) / 1e9
+    quant_gbs = quant_bytes / (q_ms * 1e-3) / 1e9
+    fp4_peak = 4.0 * peaks["bf16_sustained"]
+
+    line = {
+        "metric": METRIC, "value": prefill_tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "nvfp4", "data": "synthetic",
+        "config": {"workload": cfg.name, "N": N, "K": K, "M": M, "decode_batch": B, "parallelism": f"replicas x{world}",
+                   "l2": f"inputs larger than L2: {copies} rotating packed-weight copies "
+                         f"({copies * packed_bytes / 1e6:.0f} MB), A {2 * M * K / 1e6:.0f} MB, Y {2 * M * N / 1e6:.0f} MB",
+                   "step": "dq_prefill_quantize + dq_prefill_gemm + dq_decode_linear"},
+        "clocks": clocks,
+        "gpu_launches": 3 * args.steps,
+        "prefill": {"quant_ms": q_ms, "gemm_ms": g_ms, "gemm_tflops": gemm_tflops,
+                    "linear_tflops_per_gpu": prefill_tflops / world, "quant_gbs": quant_gbs,
+                    "quant_frac_of_hbm": quant_gbs / peaks["hbm_gbs"]},
+        "decode": {"ms": d_ms, "value": world * decode_gbs, "unit": "GB/s", "batch": B,
+                   "frac_of_measured_hbm": decode_gbs / peaks["hbm_gbs"], "frac_of_8tbs": decode_gbs / 8000.0},
+        "pack_ms": pack_ms,
+        "roofline": {"kernel": "gemm_nvfp4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(("gemm", cfg.name)),
+                     "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_sustained']} TFLOP/s); "
+                                    f"nominal dense FP4 9000"},
+        "roofline_decode": {"kernel": "gemv_lut3_kernel", "bound": "hbm", "achieved": decode_gbs,
+                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": decode_gbs / peaks["hbm_gbs"],
+                            "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)),
+                            "peak_source": f"{peaks['source']} copy bandwidth"},
+    }
+    if e2e:
+        line["e2e"] = {"value": world * flops / (e2e_p_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                       "h2d_bytes_per_step": int(2 * M * K + 2 * B * K), "d2h_bytes_per_step": int(2 * M * N + 2 * B * N),
+                       "prefill_ms": e2e_p_ms, "decode_ms": e2e_d_ms,
+                       "decode_gbs": world * dec_bytes / (e2e_d_ms * 1e-3) / 1e9}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        rows = args.ref_rows
+        W_f32 = dq_inputs.bf16_to_f32_numpy(dq_inputs.make_weight(cfg))
+        A_f32 = dq_inputs.bf16_to_f32_numpy(A_host[:rows])
+        X_f32 = dq_inputs.bf16_to_f32_numpy(X_host)
+        ref = oracle.pack_weights(W_f32)
+        tp, td = oracle_sample_run(cfg, W_f32, ref, A_f32, sa, X_f32, rows)
+        line["cpu_baseline"] = {"value": 2.0 * rows * N * K / tp / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+                                "kind": "oracle",
+                                "sample": f"{rows} of {M} prefill rows against the whole {N}x{K} layer (dequantise + fp64 "
+                                          f"matmul, {tp:.1f} s) and 1 decode token ({td:.1f} s)",
+                                "decode_gbs": (0.4375 * N * K + 2 * K + 2 * N + 4) / td / 1e9}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

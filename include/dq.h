@@ -116,6 +116,19 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
                       void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * The two stages of dq_prefill_linear as separate calls, for callers that time or
+ * overlap them: dq_prefill_quantize writes the NVFP4 activations (App. A.3 "NVFP4",
+ * static input scale) into the workspace, dq_prefill_gemm multiplies them with the
+ * handle's NVFP4 weights (Sec. 2.3).  Arguments as in dq_prefill_linear; the same
+ * M, workspace and act_global_scale must be passed to both.
+ */
+int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda,
+                        float act_global_scale, void *workspace_dev, size_t workspace_bytes,
+                        void *stream);
+int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
+                    const void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
  * Decode linear (Sec. 1.1 "memory-bound decode", App. C.2 "Kernel specification"):
  *   Y[b][n] = bf16( sum_k X[b][k] * W~[n][k] ),  W~ = s * d_b * codebook[idx],
  * a weight-only mat-vec / skinny GEMM on the handle's LUT3 weights with raw bf16

@@ -18,7 +18,8 @@ DT_FP32 = 1
 
 # every symbol include/dq.h declares
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
-           "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_decode_linear", "dq_export_canonical",
+           "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
+           "dq_decode_linear", "dq_export_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
 
 
@@ -55,6 +56,10 @@ def lib() -> C.CDLL:
         L.dq_prefill_workspace_bytes.argtypes = [vp, i64, C.POINTER(sz)]
         L.dq_prefill_linear.restype = C.c_int
         L.dq_prefill_linear.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp, sz, vp]
+        L.dq_prefill_quantize.restype = C.c_int
+        L.dq_prefill_quantize.argtypes = [vp, vp, i64, i64, C.c_float, vp, sz, vp]
+        L.dq_prefill_gemm.restype = C.c_int
+        L.dq_prefill_gemm.argtypes = [vp, i64, C.c_float, vp, i64, vp, sz, vp]
         L.dq_decode_linear.restype = C.c_int
         L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
         L.dq_export_canonical.restype = C.c_int
@@ -163,6 +168,20 @@ def prefill_linear(w: DQWeights, A: torch.Tensor, act_global_scale: float, out: 
                                    out.stride(0), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
            "dq_prefill_linear")
     return out
+
+
+def prefill_quantize(w: DQWeights, A: torch.Tensor, act_global_scale: float, workspace: torch.Tensor, stream=None):
+    """dq_prefill_quantize: stage 1 of the prefill linear (activations -> NVFP4 in the workspace)."""
+    _check(lib().dq_prefill_quantize(w.handle, A.data_ptr(), A.shape[0], A.stride(0), float(act_global_scale),
+                                     workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
+           "dq_prefill_quantize")
+
+
+def prefill_gemm(w: DQWeights, M: int, act_global_scale: float, out: torch.Tensor, workspace: torch.Tensor,
+                 stream=None):
+    """dq_prefill_gemm: stage 2 of the prefill linear (block-scaled FP4 GEMM)."""
+    _check(lib().dq_prefill_gemm(w.handle, M, float(act_global_scale), out.data_ptr(), out.stride(0),
+                                 workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)), "dq_prefill_gemm")
 
 
 def decode_linear(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:

@@ -201,32 +201,55 @@ int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_hos
     return DQ_OK;
 }
 
-int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda, float act_global_scale,
-                      void *Y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes, void *stream)
+static int prefill_checks(const dq_weights *w, int64_t M, float act_global_scale, const void *workspace_dev,
+                          size_t workspace_bytes)
 {
-    if (!valid_handle(w) || !A_dev || !Y_dev || !workspace_dev) return DQ_ERR_INVALID_ARG;
+    if (!valid_handle(w) || !workspace_dev) return DQ_ERR_INVALID_ARG;
     if (!(w->formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3))) return DQ_ERR_INVALID_ARG;
     if (M < 1 || M > (1ll << 24)) return DQ_ERR_INVALID_ARG;
     if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
-    if (lda < w->K || ldy < w->N || lda % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
-    if (!aligned(A_dev, 16) || !aligned(Y_dev, 16) || !aligned(workspace_dev, 1024)) return DQ_ERR_ALIGN;
+    if (!aligned(workspace_dev, 1024)) return DQ_ERR_ALIGN;
     size_t need = 0;
     dq_prefill_workspace_bytes(w, M, &need);
     if (workspace_bytes < need) return DQ_ERR_WORKSPACE;
-    int st = check_arch();
+    return DQ_OK;
+}
+
+int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda, float act_global_scale,
+                        void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    if (!A_dev) return DQ_ERR_INVALID_ARG;
+    int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (lda < w->K || lda % 8 != 0 || !aligned(A_dev, 16)) return DQ_ERR_ALIGN;
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
+    uint8_t *a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
+    if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, ws, a_sf, 1,
+                             reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+static int g_gemm_probe = 0;
+int dq_debug_gemm_probe(int mode) { int old = g_gemm_probe; g_gemm_probe = mode; return old; }
+
+int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
+                    const void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    if (!Y_dev) return DQ_ERR_INVALID_ARG;
+    int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (ldy < w->N || ldy % 8 != 0 || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
+    st = check_arch();
     if (st != DQ_OK) return st;
     dq::StatusWord *sw = status_word_ptr();
     if (!sw) return DQ_ERR_CUDA;
-
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
-    uint8_t *a_codes = ws;
-    uint8_t *a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
-    if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, a_codes, a_sf, 1, s) != cudaSuccess)
-        return DQ_ERR_CUDA;
+    const uint8_t *ws = reinterpret_cast<const uint8_t *>(workspace_dev);
     dq::GemmArgs g;
-    g.a_codes = a_codes;
-    g.a_sf = a_sf;
+    g.a_codes = ws;
+    g.a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
     g.w_codes = w->base + w->layout.nv_codes_off;
     g.w_sf = w->base + w->layout.nv_sf_off;
     g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
@@ -237,8 +260,22 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
     g.N = w->N;
     g.K = w->K;
     g.status = sw;
-    if (dq::launch_gemm_nvfp4(g, s) != cudaSuccess) return DQ_ERR_CUDA;
+    g.probe = g_gemm_probe;
+    if (dq::launch_gemm_nvfp4(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda, float act_global_scale,
+                      void *Y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    if (!A_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
+    int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (lda < w->K || ldy < w->N || lda % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
+    if (!aligned(A_dev, 16) || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
+    st = dq_prefill_quantize(w, A_dev, M, lda, act_global_scale, workspace_dev, workspace_bytes, stream);
+    if (st != DQ_OK) return st;
+    return dq_prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream);
 }
 
 int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,

@@ -108,8 +108,10 @@ struct GemmArgs {
     void *Y; int64_t ldy;
     int64_t M, N, K;
     StatusWord *status;
+    int probe = 0;   // timing probes: 1 = no MMA, 2 = no loads, 4 = no scale copies (results are meaningless), 8 = force the 1-CTA kernel
 };
 cudaError_t launch_gemm_nvfp4(const GemmArgs &args, cudaStream_t stream);
+cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &args, void *encode_fn, cudaStream_t stream);
 int gemm_init_driver_api();   // resolves the tensor-map encoder; 0 on success
 
 struct GemvArgs {

@@ -13,6 +13,7 @@
 #include <cuda.h>
 
 #include "dq_common.cuh"
+#include "dq_tcgen05.cuh"
 
 namespace dq {
 
@@ -33,7 +34,6 @@ constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemSfBase = 256;         // accumulator uses columns [0, 256)
 constexpr uint32_t kTmemSfBufCols = 48;       // 16 (A) + 32 (B) per stage, double buffered
-constexpr long long kWaitBudgetCycles = 4000000000ll;   // about two seconds
 
 static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment for the 128B swizzle");
 
@@ -41,110 +41,7 @@ static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment for 
 // N >> 3 at bit 17, M >> 4 at bit 24, scale-factor ids 0, K = 64
 constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait. Returns false when the budget ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t it = 0;
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if ((++it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitBudgetCycles) { *abort_flag = 1; return false; }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-// K-major operand tile, 128-byte rows, 128B swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr)
-{
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// scale atom: 32 rows x 16 bytes, unswizzled, 8-row groups 128 bytes apart
-__device__ __forceinline__ uint64_t make_desc_sf(uint32_t saddr)
-{
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (8ull << 32) | (1ull << 46);
-}
-
-__device__ __forceinline__ void tmem_cp_sf(uint32_t taddr, uint64_t desc)
-{
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
-}
-__device__ __forceinline__ void mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                         uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-        : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
+using namespace tc;
 
 // tile index -> (m block, n block): m fastest inside groups of 16 m-blocks so that
 // the CTAs running at the same time share A row-blocks and W column-blocks in L2
@@ -164,7 +61,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                   const uint8_t *__restrict__ a_sf, const uint8_t *__restrict__ w_sf,
                   const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y, int64_t ldy,
-                  int M, int N, int K, StatusWord *status)
+                  int M, int N, int K, StatusWord *status, int probe)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -222,6 +119,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t sSFA = sB + B_STAGE_BYTES;
                     const uint32_t sSFB = sSFA + SFA_STAGE_BYTES;
                     const uint32_t sf_bytes = (uint32_t)nkb * 512u;
+                    if (probe & 2) { mbar_arrive(full_bar(stage)); if (++stage == kStages) { stage = 0; phase ^= 1u; } continue; }
                     mbar_expect_tx(full_bar(stage), A_STAGE_BYTES + B_STAGE_BYTES + 3u * sf_bytes);
                     tma_load_2d(sA, &tmap_a, ks * 128, mb * BM, full_bar(stage));
                     tma_load_2d(sB, &tmap_w, ks * 128, nb * BN, full_bar(stage));
@@ -254,14 +152,14 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t sSFB = sSFA + SFA_STAGE_BYTES;
                     const uint32_t t_sfa = tmem_base + kTmemSfBase + sfbuf * kTmemSfBufCols;
                     const uint32_t t_sfb = t_sfa + 16u;
-                    for (int kb = 0; kb < nkb; ++kb) {
+                    for (int kb = 0; kb < nkb && !(probe & 4); ++kb) {
                         tmem_cp_sf(t_sfa + 4u * kb, make_desc_sf(sSFA + 512u * kb));
                         tmem_cp_sf(t_sfb + 8u * kb, make_desc_sf(sSFB + 512u * kb));
                         tmem_cp_sf(t_sfb + 8u * kb + 4u, make_desc_sf(sSFB + kKbPerStage * 512u + 512u * kb));
                     }
                     const uint64_t adesc = make_desc_sw128(sA);
                     const uint64_t bdesc = make_desc_sw128(sB);
-                    for (int kb = 0; kb < nkb; ++kb) {
+                    for (int kb = 0; kb < nkb && !(probe & 1); ++kb) {
                         // one k-step is 64 elements = 32 bytes inside the 128-byte swizzle row
                         mma_nvf4(tmem_base, adesc + 2ull * kb, bdesc + 2ull * kb, kInstrDesc, t_sfa + 4u * kb,
                                  t_sfb + 8u * kb, (ks > 0 || kb > 0) ? 1u : 0u);
@@ -367,6 +265,8 @@ int gemm_init_driver_api()
 cudaError_t launch_gemm_nvfp4(const GemmArgs &a, cudaStream_t stream)
 {
     if (gemm_init_driver_api() != 0) return cudaErrorNotSupported;
+    // more than one 128-row block: CTA pairs share the W tile; otherwise a lone CTA per tile
+    if (a.M > BM && !(a.probe & 8)) return launch_gemm_nvfp4_pair(a, reinterpret_cast<void *>(g_encode), stream);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -383,7 +283,7 @@ cudaError_t launch_gemm_nvfp4(const GemmArgs &a, cudaStream_t stream)
     const int grid = tiles < sms ? tiles : sms;
     gemm_nvfp4_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(tmap_a, tmap_w, a.a_sf, a.w_sf, a.hdr, a.act_scale,
                                                              reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy, (int)a.M,
-                                                             (int)a.N, (int)a.K, a.status);
+                                                             (int)a.N, (int)a.K, a.status, a.probe);
     return cudaGetLastError();
 }
 

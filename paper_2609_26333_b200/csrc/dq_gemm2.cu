@@ -1,0 +1,436 @@
+// NVFP4 x NVFP4 block-scaled GEMM, CTA-pair version (tcgen05 cta_group::2).
+//   Y[m][n] = bf16( s_a * s_w * sum_blk dA[m][blk] dW[n][blk] sum_{k in blk} eA[m][k] eW[n][k] )
+// (Sec. 2.3 prefill path; App. A.3 "NVFP4".)
+//
+// Two CTAs on neighbouring SMs form a cluster and compute one 256 x 256 output
+// tile per step: each CTA stages its own 128 rows of A and its own half (128
+// rows) of the W tile, so every SM reads half as many W bytes per flop as a lone
+// CTA would.  The leader CTA issues the MMAs for the pair; accumulators (128 rows
+// x 256 fp32 columns) sit in each CTA's TMEM.
+//   warp 0      : TMA producer of this CTA's operand tiles and scale atoms; all loads
+//                 signal barriers of the leader (scales and operands separately)
+//   warp 1      : (leader) tcgen05.mma; commits release the smem stage in both CTAs and
+//                 publish the accumulator to both
+//   warp 2      : (leader) tcgen05.cp of the stage's scale atoms into TMEM, one TMEM
+//                 scale buffer per smem stage.  Copies issued from their own thread
+//                 run concurrently with the MMAs; issued from the MMA thread they
+//                 serialise with them (measured: 490 us vs 240 us on 8192x17408x5120)
+//   warps 4..11 : epilogue; TMEM -> registers, TMEM released at once, then scale,
+//                 bf16 convert and global stores overlap the next tile's MMAs
+// Every wait is bounded; a wait that runs out sets DQ_ERR_TIMEOUT and all roles
+// of both CTAs leave through the common exit.
+#include <cuda.h>
+
+#include "dq_common.cuh"
+#include "dq_tcgen05.cuh"
+
+namespace dq {
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;                       // rows per CTA (pair tile: 256)
+constexpr int BN = 256;
+constexpr int kStages = 5;
+constexpr int kKbPerStage = 4;                // 64-element MMA k-steps per 256-element stage
+constexpr uint32_t A_BYTES = BM * 128;        // 16 KiB: 128 rows x 128 B of packed FP4
+constexpr uint32_t B_BYTES = (BN / 2) * 128;  // 16 KiB: this CTA's half of the W tile
+constexpr uint32_t SFA_BYTES = kKbPerStage * 512;
+constexpr uint32_t SFB_BYTES = 2 * kKbPerStage * 512;
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 38 KiB
+constexpr uint32_t SMEM_BYTES = kStages * STAGE_BYTES + 1024 + 256;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 128 + 32 * kEpiWarps;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemSfBase = 256;
+constexpr uint32_t kTmemSfBufCols = 48;      // 16 (A) + 32 (B) columns per stage
+static_assert(kTmemSfBase + kStages * kTmemSfBufCols <= kTmemCols, "scale buffers must fit in TMEM");
+static_assert(STAGE_BYTES % 1024 == 0, "stages must stay 1024-byte aligned");
+
+// dense, A/B = E2M1, K-major, UE4M3 scales, N = 256, M = 256 across the pair
+constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+constexpr uint32_t kDescHiSw128 = 64u | (1u << 14) | (2u << 29);   // SBO 1024 B, version 1, 128B swizzle
+constexpr uint32_t kDescHiSf = 8u | (1u << 14);                    // SBO 128 B, version 1, no swizzle
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_remote_u32(uint32_t cluster_addr, uint32_t v)
+{
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// pair-aware TMA tile load: data lands in this CTA, the transaction bytes are counted on `mbar_cluster`
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1,
+                                             uint32_t mbar_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(mbar_cluster) : "memory");
+}
+__device__ __forceinline__ void tmem2_cp_sf(uint32_t taddr, uint32_t lo, uint32_t hi)
+{
+    asm volatile("{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\t"
+                 "tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d;\n\t}" ::"r"(taddr), "r"(lo), "r"(hi) : "memory");
+}
+template <bool ACC>
+__device__ __forceinline__ void mma2_nvf4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t sfa,
+                                          uint32_t sfb)
+{
+    asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "setp.ne.b32 p, %7, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], da, db, %4, [%5], [%6], p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(kInstrDesc), "r"(sfa), "r"(sfb),
+                   "r"(ACC ? 1u : 0u) : "memory");
+}
+// commit all MMAs issued so far; the arrival goes to the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void mma2_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
+// commit the copies / MMAs issued so far by this thread; arrival on a barrier of this CTA only
+__device__ __forceinline__ void mma2_commit_local(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// bounded wait that also raises the partner's abort flag when it gives up
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                           uint32_t peer_abort_addr)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitBudgetCycles) {
+                *abort_flag = 1;
+                st_remote_u32(peer_abort_addr, 1u);
+                return false;
+            }
+        }
+    }
+}
+
+// pair-tile index -> (256-row block, 256-column block); m fastest inside groups of 8 so that the
+// pairs running together share W column blocks and A row blocks in L2
+__device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, int &mb, int &nb)
+{
+    constexpr int GM = 8;
+    const int per_group = GM * tiles_n;
+    const int g = t / per_group;
+    const int first_m = g * GM;
+    const int gsz = min(GM, tiles_m - first_m);
+    const int r = t - g * per_group;
+    mb = first_m + r % gsz;
+    nb = r / gsz;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                       const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
+                       const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
+                       int64_t ldy, int M, int N, int K, StatusWord *status, int probe)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + kStages * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+    auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+    auto sf_full_bar = [&](int s) { return bar_base + 8u * (3 * kStages + s); };
+    const uint32_t tmem_full_bar = bar_base + 8u * (4 * kStages);
+    const uint32_t tmem_empty_bar = bar_base + 8u * (4 * kStages + 1);
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem_gen + kStages * STAGE_BYTES + 8 * (4 * kStages + 2));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_ptr_smem + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t peer_abort = mapa(smem_u32(const_cast<int *>(abort_flag)), rank ^ 1u);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); mbar_init(sf_ready_bar(s), 1); mbar_init(sf_full_bar(s), 1); }
+        mbar_init(tmem_full_bar, 1);
+        mbar_init(tmem_empty_bar, 2 * kEpiWarps);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_ptr_smem)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers exist before anyone signals across the pair
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    const int tiles_m = (M + 2 * BM - 1) / (2 * BM);
+    const int tiles_n = (N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int katoms = K / 64;
+    const int num_ks = (katoms + kKbPerStage - 1) / kKbPerStage;
+    const int pair = blockIdx.x >> 1;
+    const int npairs = gridDim.x >> 1;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int t = pair; t < num_tiles && ok; t += npairs) {
+                int mb, nb;
+                tile_coords2(t, tiles_m, tiles_n, mb, nb);
+                const int rowblk = mb * 2 + (int)rank;            // 128-row block of A this CTA owns
+                for (int ks = 0; ks < num_ks; ++ks) {
+                    if (!mbar_wait2(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
+                    const uint32_t sA = smem_base + stage * STAGE_BYTES;
+                    const uint32_t sB = sA + A_BYTES;
+                    const uint32_t sSFA = sB + B_BYTES;
+                    const uint32_t sSFB = sSFA + SFA_BYTES;
+                    // the small scale atoms go first and have their own barrier, so that their copy
+                    // into TMEM overlaps the arrival of the operand tiles
+                    const uint32_t leader_full = mapa(full_bar(stage), 0u);
+                    const uint32_t leader_sf_full = mapa(sf_full_bar(stage), 0u);
+                    if (rank == 0) {
+                        mbar_expect_tx(sf_full_bar(stage), 2u * (SFA_BYTES + SFB_BYTES));
+                        mbar_expect_tx(full_bar(stage), 2u * (A_BYTES + B_BYTES));
+                    }
+                    if (!(probe & 2)) {
+                        tma2_load_2d(sSFA, &tmap_sfa, 0, rowblk * katoms + ks * kKbPerStage, leader_sf_full);
+                        tma2_load_2d(sSFB, &tmap_sfw, 0, (2 * nb) * katoms + ks * kKbPerStage, leader_sf_full);
+                        tma2_load_2d(sSFB + kKbPerStage * 512, &tmap_sfw, 0, (2 * nb + 1) * katoms + ks * kKbPerStage,
+                                     leader_sf_full);
+                        tma2_load_2d(sA, &tmap_a, ks * 128, rowblk * BM, leader_full);
+                        tma2_load_2d(sB, &tmap_w, ks * 128, nb * BN + (int)rank * (BN / 2), leader_full);
+                    } else if (rank == 0) {
+                        asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(sf_full_bar(stage)),
+                                     "r"(2u * (SFA_BYTES + SFB_BYTES)) : "memory");
+                        asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(full_bar(stage)),
+                                     "r"(2u * (A_BYTES + B_BYTES)) : "memory");
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------- MMA issuer (leader CTA only)
+        if (rank == 0 && lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            const uint32_t a_lo0 = ((smem_base & 0x3FFFFu) >> 4) | (1u << 16);
+            for (int t = pair; t < num_tiles && ok; t += npairs) {
+                if (!mbar_wait2(tmem_empty_bar, acc_phase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
+                tc_fence_after();
+                for (int ks = 0; ks < num_ks; ++ks) {
+                    // operand tiles of this stage are in smem and its scales are in TMEM
+                    if (!mbar_wait2(full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                    if (!mbar_wait2(sf_ready_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
+                    const uint32_t a_lo = a_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
+                    const uint32_t b_lo = a_lo + (A_BYTES >> 4);
+                    const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
+                    const uint32_t t_sfb = t_sfa + 16u;
+                    if (!(probe & 1)) {
+                        if (ks == 0) mma2_nvf4<false>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
+                        else mma2_nvf4<true>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
+#pragma unroll
+                        for (int kb = 1; kb < kKbPerStage; ++kb) {
+                            if (kb < nkb)
+                                mma2_nvf4<true>(tmem_base, a_lo + 2u * kb, b_lo + 2u * kb, kDescHiSw128, t_sfa + 4u * kb,
+                                                t_sfb + 8u * kb);
+                        }
+                    }
+                    mma2_commit_pair(empty_bar(stage));     // stage (smem and TMEM scales) reusable in both CTAs
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                mma2_commit_pair(tmem_full_bar);
+                acc_phase ^= 1u;
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------- scale copies smem -> TMEM (leader CTA only)
+        if (rank == 0 && lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            const uint32_t sf_lo0 = ((smem_base + A_BYTES + B_BYTES) & 0x3FFFFu) >> 4;
+            for (int t = pair; t < num_tiles && ok; t += npairs) {
+                for (int ks = 0; ks < num_ks; ++ks) {
+                    if (!mbar_wait2(sf_full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
+                    const uint32_t sfa_lo = sf_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
+                    const uint32_t sfb_lo = sfa_lo + (SFA_BYTES >> 4);
+                    const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
+                    const uint32_t t_sfb = t_sfa + 16u;
+                    if (!(probe & 4)) {
+#pragma unroll
+                        for (int kb = 0; kb < kKbPerStage; ++kb) {
+                            if (kb < nkb) {
+                                tmem2_cp_sf(t_sfa + 4u * kb, sfa_lo + 32u * kb, kDescHiSf);
+                                tmem2_cp_sf(t_sfb + 8u * kb, sfb_lo + 32u * kb, kDescHiSf);
+                                tmem2_cp_sf(t_sfb + 8u * kb + 4u, sfb_lo + (kKbPerStage * 512u >> 4) + 32u * kb, kDescHiSf);
+                            }
+                        }
+                    }
+                    mma2_commit_local(sf_ready_bar(stage));    // arrives once the copies have landed in both CTAs
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ epilogue
+        const int ew = warp - 4;
+        const int wq = warp & 3;                            // TMEM lane quarter this warp may read
+        const int half = ew >> 2;                           // which 128 accumulator columns
+        const float alpha = __fmul_rn(act_scale, hdr->s);
+        const uint32_t leader_tmem_empty = mapa(tmem_empty_bar, 0u);
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int t = pair; t < num_tiles && ok; t += npairs) {
+            int mb, nb;
+            tile_coords2(t, tiles_m, tiles_n, mb, nb);
+            if (!mbar_wait2(tmem_full_bar, acc_phase, abort_flag, peer_abort)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(half * 128);
+            uint32_t v0[32], v1[32], v2[32], v3[32];
+            tmem_ld32(taddr, v0);
+            tmem_ld32(taddr + 32u, v1);
+            tmem_ld32(taddr + 64u, v2);
+            tmem_ld32(taddr + 96u, v3);
+            tmem_ld_wait();
+            // the accumulator is in registers: hand TMEM back before converting and storing
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(leader_tmem_empty);
+            acc_phase ^= 1u;
+
+            const int row = (mb * 2 + (int)rank) * BM + wq * 32 + lane;
+            const int col0 = nb * BN + half * 128;
+            if (row < M && !(probe & 32)) {
+                __nv_bfloat16 *yrow = Y + (int64_t)row * ldy + col0;
+                auto store32 = [&](const uint32_t (&v)[32], int c) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (col0 + c + q * 8 < N) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]) * alpha, __uint_as_float(v[8 * q + 1]) * alpha);
+                            o.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]) * alpha, __uint_as_float(v[8 * q + 3]) * alpha);
+                            o.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]) * alpha, __uint_as_float(v[8 * q + 5]) * alpha);
+                            o.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]) * alpha, __uint_as_float(v[8 * q + 7]) * alpha);
+                            *reinterpret_cast<uint4 *>(yrow + c + q * 8) = o;
+                        }
+                    }
+                };
+                store32(v0, 0);
+                store32(v1, 32);
+                store32(v2, 64);
+                store32(v3, 96);
+            }
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // nobody leaves while the partner may still signal its barriers
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);       // let copies in flight land
+        if (threadIdx.x == 0) {
+            atomicExch(&status->status, (int)DQ_ERR_TIMEOUT);
+            atomicExch(&status->detail, 0x20000 | (int)blockIdx.x);
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool make_codes_tmap2(EncodeTiledFn enc, CUtensorMap *tm, const void *ptr, int64_t rows, int64_t K, uint32_t box_rows)
+{
+    cuuint64_t gdim[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)(K / 2)};
+    cuuint32_t box[2] = {128u, box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), gdim, gstride, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// scale atoms as a matrix of 512-byte rows (128 x uint32); box = 4 consecutive k atoms
+bool make_sf_tmap(EncodeTiledFn enc, CUtensorMap *tm, const void *ptr, int64_t atoms)
+{
+    cuuint64_t gdim[2] = {128u, (cuuint64_t)atoms};
+    cuuint64_t gstride[1] = {512u};
+    cuuint32_t box[2] = {128u, (cuuint32_t)kKbPerStage};
+    cuuint32_t estr[2] = {1u, 1u};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(ptr), gdim, gstride, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStream_t stream)
+{
+    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(encode_fn);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int64_t katoms = a.K / 64;
+    CUtensorMap tmap_a, tmap_w, tmap_sfa, tmap_sfw;
+    if (!make_codes_tmap2(enc, &tmap_a, a.a_codes, a.M, a.K, BM)) return cudaErrorInvalidValue;
+    if (!make_codes_tmap2(enc, &tmap_w, a.w_codes, a.N, a.K, BN / 2)) return cudaErrorInvalidValue;
+    if (!make_sf_tmap(enc, &tmap_sfa, a.a_sf, ((a.M + 127) / 128) * katoms)) return cudaErrorInvalidValue;
+    if (!make_sf_tmap(enc, &tmap_sfw, a.w_sf, ((a.N + 255) / 256) * 2 * katoms)) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
+    int pairs = sms / 2;
+    if (tiles < pairs) pairs = tiles;
+    gemm_nvfp4_pair_kernel<<<2 * pairs, kThreads, SMEM_BYTES, stream>>>(
+        tmap_a, tmap_w, tmap_sfa, tmap_sfw, a.hdr, a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy,
+        (int)a.M, (int)a.N, (int)a.K, a.status, a.probe);
+    return cudaGetLastError();
+}
+
+}  // namespace dq
