@@ -152,14 +152,15 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
             return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_LUT3) {
-        if (dq::launch_pack_lut3(W_dev, w_dtype, N, K, ldw, hdr,
-                                 reinterpret_cast<uint32_t *>(base + L.lut_planes_off), base + L.lut_sf_off, s) !=
-            cudaSuccess)
+        if (L.lut_bytes != (size_t)N * K / 16 * 7) {       // partial last slice: padding must read as zero
+            if (cudaMemsetAsync(base + L.lut_off, 0, L.lut_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+        }
+        if (dq::launch_pack_lut3(W_dev, w_dtype, N, K, ldw, hdr, base + L.lut_off, s) != cudaSuccess)
             return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
-        if (dq::launch_autocast(hdr, reinterpret_cast<const uint32_t *>(base + L.lut_planes_off), base + L.lut_sf_off,
-                                N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) != cudaSuccess)
+        if (dq::launch_autocast(hdr, base + L.lut_off, N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
+            cudaSuccess)
             return DQ_ERR_CUDA;
     }
     dq_weights *w = new (std::nothrow) dq_weights;
@@ -289,8 +290,9 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
     int st = check_arch();
     if (st != DQ_OK) return st;
     dq::GemvArgs g;
-    g.planes = reinterpret_cast<const uint32_t *>(w->base + w->layout.lut_planes_off);
-    g.sf = w->base + w->layout.lut_sf_off;
+    g.lut = w->base + w->layout.lut_off;
+    g.status = status_word_ptr();
+    if (!g.status) return DQ_ERR_CUDA;
     g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
     g.X = X_dev;
     g.ldx = ldx;
@@ -319,8 +321,7 @@ int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, v
     }
     if (format == DQ_FMT_LUT3) {
         if (!(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
-        if (dq::launch_export_lut3(hdr, reinterpret_cast<const uint32_t *>(w->base + w->layout.lut_planes_off),
-                                   w->base + w->layout.lut_sf_off, w->N, w->K,
+        if (dq::launch_export_lut3(hdr, w->base + w->layout.lut_off, w->N, w->K,
                                    reinterpret_cast<uint32_t *>(codes_dev), reinterpret_cast<uint8_t *>(scales_dev),
                                    global_scale_dev, s) != cudaSuccess)
             return DQ_ERR_CUDA;

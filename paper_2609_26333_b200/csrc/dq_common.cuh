@@ -16,7 +16,6 @@ constexpr int kBlock = 16;            // weights per block scale (App. A.3)
 constexpr int kSfAtomRows = 128;      // rows of one scale-factor atom of the block-scaled MMA
 constexpr int kSfAtomBytes = 512;     // 128 rows x 4 scales (64 k)
 constexpr int kSfRowPad = 256;        // NVFP4 scale tiles padded to the GEMM's N tile
-constexpr int kLutChunk = 128;        // weights per LUT3 device chunk (3 planes x 4 words)
 
 // Device header at the start of the packed buffer (1 KiB reserved).
 struct PackedHeader {
@@ -32,11 +31,30 @@ struct PackedHeader {
 };
 constexpr size_t kHeaderBytes = 1024;
 
+// LUT3 device layout: the weights of one row are cut into slices of 1024 (one per warp of the
+// decode kernel); slice s of row r is one block of 448 bytes:
+//   [plane 0: 32 words][plane 1: 32 words][plane 2: 32 words][scales: 64 signed E4M3 bytes]
+// i.e. 3 bit-plane words + 2 scale bytes per lane, 3.5 bit per weight.  A partial last slice is
+// zero padded (zero scales, so the padding contributes nothing).
+constexpr int kLutSlice = 1024;
+constexpr int kLutBlockBytes = 448;
+constexpr int kLutScaleOff = 384;
+__host__ __device__ inline int64_t lut_slices(int64_t K) { return (K + kLutSlice - 1) / kLutSlice; }
+// word j (32 weights) of plane p in row r; K/32 words per row
+__host__ __device__ inline size_t lut_word_offset(int64_t r, int64_t j, int p, int64_t K)
+{
+    return (size_t)(r * lut_slices(K) + j / 32) * kLutBlockBytes + (size_t)p * 128 + (size_t)(j % 32) * 4;
+}
+// scale of 16-block b in row r
+__host__ __device__ inline size_t lut_scale_offset(int64_t r, int64_t b, int64_t K)
+{
+    return (size_t)(r * lut_slices(K) + b / 64) * kLutBlockBytes + kLutScaleOff + (size_t)(b % 64);
+}
+
 struct PackedLayout {
     size_t nv_codes_off = 0, nv_codes_bytes = 0;     // uint8[N][K/2]
     size_t nv_sf_off = 0, nv_sf_bytes = 0;           // [ceil(N/256)*2][K/64][512] MMA scale layout
-    size_t lut_planes_off = 0, lut_planes_bytes = 0; // uint32[N][K/128][3][4]
-    size_t lut_sf_off = 0, lut_sf_bytes = 0;         // uint8[N][K/16] signed E4M3
+    size_t lut_off = 0, lut_bytes = 0;               // [N][ceil(K/1024)] blocks of kLutBlockBytes (see below)
     size_t total = 0;
 };
 
@@ -55,12 +73,9 @@ inline PackedLayout packed_layout(int64_t N, int64_t K, unsigned formats)
         off = align_up(off + L.nv_sf_bytes, 1024);
     }
     if (formats & (DQ_FMT_LUT3 | DQ_FMT_NVFP4_FROM_LUT3)) {
-        L.lut_planes_off = off;
-        L.lut_planes_bytes = (size_t)N * K / 8 * 3;
-        off = align_up(off + L.lut_planes_bytes, 1024);
-        L.lut_sf_off = off;
-        L.lut_sf_bytes = (size_t)N * (K / kBlock);
-        off = align_up(off + L.lut_sf_bytes, 1024);
+        L.lut_off = off;
+        L.lut_bytes = (size_t)N * lut_slices(K) * kLutBlockBytes;
+        off = align_up(off + L.lut_bytes, 1024);
     }
     L.total = off;
     return L;
@@ -76,6 +91,18 @@ __host__ __device__ inline size_t sf_swizzled_offset(int64_t r, int64_t b, int64
     return (size_t)atom * 512 + (size_t)(rr % 32) * 16 + (size_t)(rr / 32) * 4 + (size_t)(b % 4);
 }
 
+// LUT3 device bit order.  The planes keep the (N, 3, K/32) int32 shape of App. C.2; inside a
+// word the 32 weights are permuted so that the decode kernel can assemble the six index bits of
+// two neighbouring weights (2q, 2q+1) into one byte with two bitwise selects:
+//   q = 4g + j  ->  plane p holds bit p of weight 2q+e at position (8j + 2g + e + 2p) mod 32.
+// Rotating the three plane words right by 2g and taking bits {0,1} / {2,3} / {4,5} of byte j from
+// planes 0 / 1 / 2 yields  b0a b0b b1a b1b b2a b2b  in the low six bits of that byte.
+__host__ __device__ inline int lut3_bitpos(int plane, int i)
+{
+    const int q = i >> 1, e = i & 1;
+    return (8 * (q & 3) + 2 * (q >> 2) + e + 2 * plane) & 31;
+}
+
 // Device status word: [0] = dq_status, [1] = detail.
 struct StatusWord { int status; int detail; };
 
@@ -86,13 +113,13 @@ cudaError_t launch_absmax(const void *W, int w_dtype, int64_t N, int64_t K, int6
 cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
                               const PackedHeader *hdr, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream);
 cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
-                             const PackedHeader *hdr, uint32_t *planes_dev, uint8_t *lut_sf, cudaStream_t stream);
-cudaError_t launch_autocast(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+                             const PackedHeader *hdr, uint8_t *lut_dev, cudaStream_t stream);
+cudaError_t launch_autocast(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                             int64_t K, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream);
 cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, const uint8_t *sf_swizzled, int64_t N,
                                 int64_t K, uint8_t *codes_out, uint8_t *scales_out, float *s_out,
                                 cudaStream_t stream);
-cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                                int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
                                cudaStream_t stream);
 // Activation quantiser: codes row-major [M][K/2]; scales either in the MMA layout
@@ -115,7 +142,8 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &args, void *encode_fn, cudaSt
 int gemm_init_driver_api();   // resolves the tensor-map encoder; 0 on success
 
 struct GemvArgs {
-    const uint32_t *planes; const uint8_t *sf; const PackedHeader *hdr;
+    const uint8_t *lut; const PackedHeader *hdr;          // LUT3 blocks (planes + scales)
+    StatusWord *status = nullptr;
     const void *X; int64_t ldx; int64_t B;
     void *Y; int64_t ldy;
     int64_t N, K;

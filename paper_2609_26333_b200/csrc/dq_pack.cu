@@ -198,7 +198,7 @@ cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, 
 // One thread quantises 32 consecutive weights (two 16-blocks) and emits one word of each bit-plane.
 template <bool FP32IN>
 __global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ldw, const PackedHeader *hdr,
-                                 uint32_t *planes, uint8_t *lut_sf)
+                                 uint8_t *lut)
 {
     const int64_t nw = K / 32;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -223,7 +223,7 @@ __global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ld
         }
         uint32_t d8 = f32_to_e4m3(__fmul_rn(m, rc6));
         if ((d8 & 0x7Fu) == 0u) d8 = 0u;
-        lut_sf[r * (K / 16) + j * 2 + h] = (uint8_t)d8;
+        lut[lut_scale_offset(r, j * 2 + h, K)] = (uint8_t)d8;
         const float rr = (d8 != 0u) ? __frcp_rn(__fmul_rn(s, e4m3_to_f32(d8))) : 0.0f;
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -234,24 +234,25 @@ __global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ld
 #pragma unroll
                 for (int l = 0; l < 7; ++l) idx += (y > T[l]) ? 1 : 0;
             }
-            const int bit = h * 16 + q;
-            p0 |= (uint32_t)(idx & 1) << bit;
-            p1 |= (uint32_t)((idx >> 1) & 1) << bit;
-            p2 |= (uint32_t)((idx >> 2) & 1) << bit;
+            const int i = h * 16 + q;
+            p0 |= (uint32_t)(idx & 1) << lut3_bitpos(0, i);
+            p1 |= (uint32_t)((idx >> 1) & 1) << lut3_bitpos(1, i);
+            p2 |= (uint32_t)((idx >> 2) & 1) << lut3_bitpos(2, i);
         }
     }
-    // device layout: [row][K/128 chunks][plane][4 words]
-    uint32_t *dst = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
-    dst[0] = p0; dst[4] = p1; dst[8] = p2;
+    // device layout: 448-byte blocks per (row, 1024-weight slice); bit order inside a word per lut3_bitpos
+    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 0, K)) = p0;
+    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 1, K)) = p1;
+    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 2, K)) = p2;
 }
 
 cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
-                             const PackedHeader *hdr, uint32_t *planes_dev, uint8_t *lut_sf, cudaStream_t stream)
+                             const PackedHeader *hdr, uint8_t *lut_dev, cudaStream_t stream)
 {
     const int64_t total = N * (K / 32);
     const unsigned blocks = (unsigned)((total + 127) / 128);
-    if (w_dtype == DQ_DT_FP32) pack_lut3_kernel<true><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, planes_dev, lut_sf);
-    else pack_lut3_kernel<false><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, planes_dev, lut_sf);
+    if (w_dtype == DQ_DT_FP32) pack_lut3_kernel<true><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+    else pack_lut3_kernel<false><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
     return cudaGetLastError();
 }
 
@@ -259,7 +260,7 @@ cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, i
 
 // NVFP4 view of the LUT3 codes (Sec. 2.3): level -> nearest E2M1 value, element signs
 // flipped under a negative block scale, block scale |d|, same tensor scale.
-__global__ void autocast_kernel(const PackedHeader *hdr, const uint32_t *planes, const uint8_t *lut_sf, int64_t N,
+__global__ void autocast_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
                                 int64_t K, uint8_t *codes, uint8_t *sf)
 {
     const int64_t nw = K / 32;
@@ -267,17 +268,19 @@ __global__ void autocast_kernel(const PackedHeader *hdr, const uint32_t *planes,
     if (i >= N * nw) return;
     const int64_t r = i / nw, j = i % nw;
     const uint32_t amap = hdr->autocast_map;
-    const uint32_t *src = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
-    const uint32_t p0 = src[0], p1 = src[4], p2 = src[8];
+    const uint32_t p0 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 0, K));
+    const uint32_t p1 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 1, K));
+    const uint32_t p2 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 2, K));
     uint32_t out[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const uint32_t d8 = lut_sf[r * (K / 16) + j * 2 + h];
+        const uint32_t d8 = lut[lut_scale_offset(r, j * 2 + h, K)];
         sf[sf_swizzled_offset(r, j * 2 + h, K)] = (uint8_t)(d8 & 0x7Fu);
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int bit = h * 16 + q;
-            const uint32_t idx = ((p0 >> bit) & 1u) | (((p1 >> bit) & 1u) << 1) | (((p2 >> bit) & 1u) << 2);
+            const uint32_t idx = ((p0 >> lut3_bitpos(0, bit)) & 1u) | (((p1 >> lut3_bitpos(1, bit)) & 1u) << 1) |
+                                 (((p2 >> lut3_bitpos(2, bit)) & 1u) << 2);
             uint32_t c = (amap >> (4 * idx)) & 0xFu;
             if ((d8 & 0x80u) && (c & 0x7u)) c ^= 0x8u;
             if (d8 == 0u) c = 0u;
@@ -287,12 +290,11 @@ __global__ void autocast_kernel(const PackedHeader *hdr, const uint32_t *planes,
     *reinterpret_cast<uint4 *>(codes + r * (K / 2) + j * 16) = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
-cudaError_t launch_autocast(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+cudaError_t launch_autocast(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                             int64_t K, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream)
 {
     const int64_t total = N * (K / 32);
-    autocast_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(hdr, planes_dev, lut_sf, N, K, codes,
-                                                                         sf_swizzled);
+    autocast_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(hdr, lut_dev, N, K, codes, sf_swizzled);
     return cudaGetLastError();
 }
 
@@ -321,7 +323,7 @@ cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, c
     return cudaGetLastError();
 }
 
-__global__ void export_lut3_kernel(const PackedHeader *hdr, const uint32_t *planes, const uint8_t *lut_sf, int64_t N,
+__global__ void export_lut3_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
                                    int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out)
 {
     const int64_t nw = K / 32;
@@ -329,19 +331,24 @@ __global__ void export_lut3_kernel(const PackedHeader *hdr, const uint32_t *plan
     if (i == 0 && s_out) *s_out = hdr->s;
     if (i >= N * nw) return;
     const int64_t r = i / nw, j = i % nw;
-    const uint32_t *src = planes + ((r * (K / 128) + j / 4) * 3) * 4 + (j % 4);
 #pragma unroll
-    for (int p = 0; p < 3; ++p) planes_out[(r * 3 + p) * nw + j] = src[4 * p];
-    scales_out[r * (K / 16) + 2 * j] = lut_sf[r * (K / 16) + 2 * j];
-    scales_out[r * (K / 16) + 2 * j + 1] = lut_sf[r * (K / 16) + 2 * j + 1];
+    for (int p = 0; p < 3; ++p) {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, p, K));
+        uint32_t c = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) c |= ((w >> lut3_bitpos(p, i)) & 1u) << i;      // canonical: LSB-first
+        planes_out[(r * 3 + p) * nw + j] = c;
+    }
+    scales_out[r * (K / 16) + 2 * j] = lut[lut_scale_offset(r, 2 * j, K)];
+    scales_out[r * (K / 16) + 2 * j + 1] = lut[lut_scale_offset(r, 2 * j + 1, K)];
 }
 
-cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint32_t *planes_dev, const uint8_t *lut_sf, int64_t N,
+cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                                int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
                                cudaStream_t stream)
 {
     const int64_t total = N * (K / 32);
-    export_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, planes_dev, lut_sf, N, K, planes_out,
+    export_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, lut_dev, N, K, planes_out,
                                                                             scales_out, s_out);
     return cudaGetLastError();
 }
