@@ -129,6 +129,27 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
                     const void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * dq_prefill_linear without a caller-provided workspace.  (The paper has no counterpart: this
+ * entry point exists for integration, not for the method.)
+ * It is meant for callers that cannot allocate device memory where they call from -- an engine
+ * whose memory pool already owns all of HBM, code running inside another process's allocator
+ * regime, or a thread that must not hit the device-wide synchronisation inside cudaMalloc and
+ * cudaFree.  The scratch is an array built into the library (8 MiB per GPU that loads it, held
+ * until the process exits); no cudaMalloc, cudaFree or allocating library routine is called.
+ * Limit: dq_prefill_workspace_bytes(w, M) must not exceed 8 MiB (8388608 bytes), i.e. roughly
+ * M * K <= 14.9 M elements; larger problems return DQ_ERR_WORKSPACE and nothing is launched.
+ * The first call on a device looks up the array's device address (once per device, with that
+ * device current); make that first call before starting any stream capture.
+ * All calls on a device share the one array: two calls whose GPU work overlaps (different
+ * streams without ordering) race on it and give wrong results; calls ordered on one stream, or
+ * by events, are safe.  The array keeps the previous call's contents; the call clears the part
+ * it reads without rewriting.
+ * Other arguments, results and status codes as dq_prefill_linear.
+ */
+int dq_prefill_linear_static(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda,
+                             float act_global_scale, void *Y_dev, int64_t ldy, void *stream);
+
+/*
  * Decode linear (Sec. 1.1 "memory-bound decode", App. C.2 "Kernel specification"):
  *   Y[b][n] = bf16( sum_k X[b][k] * W~[n][k] ),  W~ = s * d_b * codebook[idx],
  * a weight-only mat-vec / skinny GEMM on the handle's LUT3 weights with raw bf16

@@ -19,6 +19,7 @@ DT_FP32 = 1
 # every symbol include/dq.h declares
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
+           "dq_prefill_linear_static",
            "dq_decode_linear", "dq_export_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
 
@@ -60,6 +61,8 @@ def lib() -> C.CDLL:
         L.dq_prefill_quantize.argtypes = [vp, vp, i64, i64, C.c_float, vp, sz, vp]
         L.dq_prefill_gemm.restype = C.c_int
         L.dq_prefill_gemm.argtypes = [vp, i64, C.c_float, vp, i64, vp, sz, vp]
+        L.dq_prefill_linear_static.restype = C.c_int
+        L.dq_prefill_linear_static.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp]
         L.dq_decode_linear.restype = C.c_int
         L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
         L.dq_export_canonical.restype = C.c_int
@@ -167,6 +170,23 @@ def prefill_linear(w: DQWeights, A: torch.Tensor, act_global_scale: float, out: 
     _check(lib().dq_prefill_linear(w.handle, A.data_ptr(), M, A.stride(0), float(act_global_scale), out.data_ptr(),
                                    out.stride(0), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
            "dq_prefill_linear")
+    return out
+
+
+def prefill_linear_static(w: DQWeights, A: torch.Tensor, act_global_scale: float, out: torch.Tensor = None,
+                          stream=None) -> torch.Tensor:
+    """dq_prefill_linear_static: the prefill linear on the library's built-in 8 MiB scratch.
+
+    For callers that cannot allocate device memory at the call site (all HBM owned by a pool,
+    foreign allocator, no tolerance for cudaMalloc's synchronisation).  Calls that overlap on
+    the GPU race on the shared scratch."""
+    assert A.is_cuda and A.dtype == torch.bfloat16 and A.dim() == 2 and A.stride(1) == 1 and A.shape[1] == w.K
+    M = A.shape[0]
+    if out is None:
+        out = torch.empty(M, w.N, dtype=torch.bfloat16, device=A.device)
+    _check(lib().dq_prefill_linear_static(w.handle, A.data_ptr(), M, A.stride(0), float(act_global_scale),
+                                          out.data_ptr(), out.stride(0), _stream_ptr(stream)),
+           "dq_prefill_linear_static")
     return out
 
 
