@@ -37,8 +37,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum);
 # see profiles/ for the captures these come from.  None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {
-    ("gemm", "c3_gate_up27b"): None,
-    ("gemv", "c3_gate_up27b"): None,
+    ("gemm", "c3_gate_up27b"): 221.4e6 + 235.2e6,     # profiles/launch_list_c3_gate_up27b.md
+    ("gemv", "c3_gate_up27b"): 39.04e6,
 }
 
 
@@ -54,7 +54,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
 
-    def __init__(self, device_index: int, period_s: float = 0.05):
+    def __init__(self, device_index: int, period_s: float = 0.01):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -143,7 +143,7 @@ def run_reference(args, cfg):
     A_f32 = dq_inputs.bf16_to_f32_numpy(A)
     X_f32 = dq_inputs.bf16_to_f32_numpy(dq_inputs.make_activations(cfg, 1, salt=2))
     ref = oracle.pack_weights(W_f32)
-    for _ in range(args.warmup):
+    for _ in range(min(args.warmup, 2)):
         oracle_sample_run(cfg, W_f32, ref, A_f32, sa, X_f32, rows)
     tp = td = 0.0
     t0 = time.perf_counter()
@@ -171,8 +171,8 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(dq_inputs.CONFIGS))
     ap.add_argument("--mnk", default=None, help="M,N,K of an ad-hoc Gaussian layer (profiling small cases)")
     ap.add_argument("--impl", default="dq", choices=["dq", "reference"])
@@ -350,7 +350,7 @@ def main():
         "decode": {"ms": d_ms, "value": world * decode_gbs, "unit": "GB/s", "batch": B,
                    "frac_of_measured_hbm": decode_gbs / peaks["hbm_gbs"], "frac_of_8tbs": decode_gbs / 8000.0},
         "pack_ms": pack_ms,
-        "roofline": {"kernel": "gemm_nvfp4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
+        "roofline": {"kernel": "gemm_nvfp4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(("gemm", cfg.name)),
                      "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_sustained']} TFLOP/s); "
