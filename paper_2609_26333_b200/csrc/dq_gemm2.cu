@@ -11,12 +11,12 @@
 //                 signal barriers of the leader (scales and operands separately)
 //   warp 1      : (leader) tcgen05.mma; commits release the smem stage in both CTAs and
 //                 publish the accumulator to both
-//   warp 2      : (leader) tcgen05.cp of the stage's scale atoms into TMEM, one TMEM
-//                 scale buffer per smem stage.  Copies issued from their own thread
+//   warps 2, 3  : (leader) tcgen05.cp of the stage's scale atoms into TMEM, one TMEM
+//                 scale buffer per smem stage; the two warps take alternate k-steps.  Copies issued from their own thread
 //                 run concurrently with the MMAs; issued from the MMA thread they
 //                 serialise with them (measured: 490 us vs 240 us on 8192x17408x5120)
-//   warps 4..11 : epilogue; TMEM -> registers, TMEM released at once, then scale,
-//                 bf16 convert and global stores overlap the next tile's MMAs
+//   warps 4..11 : epilogue; TMEM -> registers, TMEM released at once, then scale, bf16
+//                 convert, swizzled smem staging and TMA stores overlap the next tile's MMAs
 // Every wait is bounded; a wait that runs out sets DQ_ERR_TIMEOUT and all roles
 // of both CTAs leave through the common exit.
 #include <cuda.h>
@@ -39,7 +39,10 @@ constexpr uint32_t B_BYTES = (BN / 2) * 128;  // 16 KiB: this CTA's half of the 
 constexpr uint32_t SFA_BYTES = kKbPerStage * 512;
 constexpr uint32_t SFB_BYTES = 2 * kKbPerStage * 512;
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 38 KiB
-constexpr uint32_t SMEM_BYTES = kStages * STAGE_BYTES + 1024 + 256;
+constexpr uint32_t STG_WARP_BYTES = 32 * 128;                                  // 32 rows x 64 bf16, one TMA-store box
+constexpr uint32_t STG_OFF = kStages * STAGE_BYTES;                           // epilogue staging, 1024-byte aligned
+constexpr uint32_t BAR_OFF = STG_OFF + 8 * STG_WARP_BYTES;
+constexpr uint32_t SMEM_BYTES = BAR_OFF + 1024 + 256;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 128 + 32 * kEpiWarps;
 constexpr uint32_t kTmemCols = 512;
@@ -100,6 +103,17 @@ __device__ __forceinline__ void mma2_nvf4(uint32_t d_tmem, uint32_t a_lo, uint32
                  ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(kInstrDesc), "r"(sfa), "r"(sfb),
                    "r"(ACC ? 1u : 0u) : "memory");
 }
+// TMA store of one staged box (shared -> global); out-of-range rows / columns are clipped by the hardware
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *tmap, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tmap), "r"(src), "r"(c0), "r"(c1) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 // commit all MMAs issued so far; the arrival goes to the barrier at this offset in both CTAs of the pair
 __device__ __forceinline__ void mma2_commit_pair(uint32_t bar)
 {
@@ -150,20 +164,20 @@ __device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, in
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
-                       const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
+                       const __grid_constant__ CUtensorMap tmap_y, const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
                        int64_t ldy, int M, int N, int K, StatusWord *status, int probe)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t bar_base = smem_base + kStages * STAGE_BYTES;
+    const uint32_t bar_base = smem_base + BAR_OFF;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
     auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
     auto sf_full_bar = [&](int s) { return bar_base + 8u * (3 * kStages + s); };
     const uint32_t tmem_full_bar = bar_base + 8u * (4 * kStages);
     const uint32_t tmem_empty_bar = bar_base + 8u * (4 * kStages + 1);
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem_gen + kStages * STAGE_BYTES + 8 * (4 * kStages + 2));
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem_gen + BAR_OFF + 8 * (4 * kStages + 2));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_ptr_smem + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -276,32 +290,38 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 acc_phase ^= 1u;
             }
         }
-    } else if (warp == 2) {
+    } else if (warp == 2 || warp == 3) {
         // ------------------------------- scale copies smem -> TMEM (leader CTA only)
+        // One thread can issue only about one copy per 30 ns, and a stage needs 12 of them plus the
+        // barrier round trips, which is more than the 0.4 us its MMAs take; so two threads take
+        // alternate stages (warp 2 the even k-steps, warp 3 the odd ones).
         if (rank == 0 && lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             const uint32_t sf_lo0 = ((smem_base + A_BYTES + B_BYTES) & 0x3FFFFu) >> 4;
+            uint32_t step = 0;
             for (int t = pair; t < num_tiles && ok; t += npairs) {
-                for (int ks = 0; ks < num_ks; ++ks) {
-                    if (!mbar_wait2(sf_full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
-                    tc_fence_after();
-                    const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
-                    const uint32_t sfa_lo = sf_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
-                    const uint32_t sfb_lo = sfa_lo + (SFA_BYTES >> 4);
-                    const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
-                    const uint32_t t_sfb = t_sfa + 16u;
-                    if (!(probe & 4)) {
+                for (int ks = 0; ks < num_ks; ++ks, ++step) {
+                    if ((step & 1u) == (uint32_t)(warp - 2)) {
+                        if (!mbar_wait2(sf_full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                        tc_fence_after();
+                        const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
+                        const uint32_t sfa_lo = sf_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
+                        const uint32_t sfb_lo = sfa_lo + (SFA_BYTES >> 4);
+                        const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
+                        const uint32_t t_sfb = t_sfa + 16u;
+                        if (!(probe & 4)) {
 #pragma unroll
-                        for (int kb = 0; kb < kKbPerStage; ++kb) {
-                            if (kb < nkb) {
-                                tmem2_cp_sf(t_sfa + 4u * kb, sfa_lo + 32u * kb, kDescHiSf);
-                                tmem2_cp_sf(t_sfb + 8u * kb, sfb_lo + 32u * kb, kDescHiSf);
-                                tmem2_cp_sf(t_sfb + 8u * kb + 4u, sfb_lo + (kKbPerStage * 512u >> 4) + 32u * kb, kDescHiSf);
+                            for (int kb = 0; kb < kKbPerStage; ++kb) {
+                                if (kb < nkb) {
+                                    tmem2_cp_sf(t_sfa + 4u * kb, sfa_lo + 32u * kb, kDescHiSf);
+                                    tmem2_cp_sf(t_sfb + 8u * kb, sfb_lo + 32u * kb, kDescHiSf);
+                                    tmem2_cp_sf(t_sfb + 8u * kb + 4u, sfb_lo + (kKbPerStage * 512u >> 4) + 32u * kb, kDescHiSf);
+                                }
                             }
                         }
+                        mma2_commit_local(sf_ready_bar(stage));    // arrives once the copies have landed in both CTAs
                     }
-                    mma2_commit_local(sf_ready_bar(stage));    // arrives once the copies have landed in both CTAs
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -333,29 +353,36 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             if (lane == 0) mbar_arrive_remote(leader_tmem_empty);
             acc_phase ^= 1u;
 
-            const int row = (mb * 2 + (int)rank) * BM + wq * 32 + lane;
+            // bf16 rows go through a swizzled staging box (32 rows x 64 columns per warp) and leave with
+            // a TMA store, so that global memory sees full 128-byte lines instead of 16-byte pieces
+            const int row0 = (mb * 2 + (int)rank) * BM + wq * 32;
             const int col0 = nb * BN + half * 128;
-            if (row < M && !(probe & 32)) {
-                __nv_bfloat16 *yrow = Y + (int64_t)row * ldy + col0;
-                auto store32 = [&](const uint32_t (&v)[32], int c) {
+            if (!(probe & 32)) {
+                const uint32_t stg = smem_base + STG_OFF + (uint32_t)ew * STG_WARP_BYTES;
+                const uint32_t my_row = stg + (uint32_t)lane * 128u;
+                const uint32_t sw = (uint32_t)(lane & 7);
+                auto stage_box = [&](const uint32_t (&lo)[32], const uint32_t (&hi)[32], int box) {
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer free again
+                    __syncwarp();
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (col0 + c + q * 8 < N) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]) * alpha, __uint_as_float(v[8 * q + 1]) * alpha);
-                            o.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]) * alpha, __uint_as_float(v[8 * q + 3]) * alpha);
-                            o.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]) * alpha, __uint_as_float(v[8 * q + 5]) * alpha);
-                            o.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]) * alpha, __uint_as_float(v[8 * q + 7]) * alpha);
-                            *reinterpret_cast<uint4 *>(yrow + c + q * 8) = o;
-                        }
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t (&v)[32] = (c < 4) ? lo : hi;
+                        const int o = (c & 3) * 8;
+                        sts_v4(my_row + (((uint32_t)c ^ sw) << 4),
+                               pack_bf16x2(__uint_as_float(v[o + 0]) * alpha, __uint_as_float(v[o + 1]) * alpha),
+                               pack_bf16x2(__uint_as_float(v[o + 2]) * alpha, __uint_as_float(v[o + 3]) * alpha),
+                               pack_bf16x2(__uint_as_float(v[o + 4]) * alpha, __uint_as_float(v[o + 5]) * alpha),
+                               pack_bf16x2(__uint_as_float(v[o + 6]) * alpha, __uint_as_float(v[o + 7]) * alpha));
                     }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0 && row0 < M && col0 + box * 64 < N) tma_store_2d(&tmap_y, stg, col0 + box * 64, row0);
                 };
-                store32(v0, 0);
-                store32(v1, 32);
-                store32(v2, 64);
-                store32(v3, 96);
+                stage_box(v0, v1, 0);
+                stage_box(v2, v3, 1);
             }
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // all stores of this warp done
     }
 
     __syncwarp();
@@ -403,6 +430,18 @@ bool make_sf_tmap(EncodeTiledFn enc, CUtensorMap *tm, const void *ptr, int64_t a
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 output matrix [M][N] with row stride ldy; box = 64 columns x 32 rows, 128B swizzle
+bool make_y_tmap(EncodeTiledFn enc, CUtensorMap *tm, void *ptr, int64_t M, int64_t N, int64_t ldy)
+{
+    cuuint64_t gdim[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t gstride[1] = {(cuuint64_t)ldy * 2u};
+    cuuint32_t box[2] = {64u, 32u};
+    cuuint32_t estr[2] = {1u, 1u};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStream_t stream)
@@ -416,11 +455,12 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
         attr_set = true;
     }
     const int64_t katoms = a.K / 64;
-    CUtensorMap tmap_a, tmap_w, tmap_sfa, tmap_sfw;
+    CUtensorMap tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y;
     if (!make_codes_tmap2(enc, &tmap_a, a.a_codes, a.M, a.K, BM)) return cudaErrorInvalidValue;
     if (!make_codes_tmap2(enc, &tmap_w, a.w_codes, a.N, a.K, BN / 2)) return cudaErrorInvalidValue;
     if (!make_sf_tmap(enc, &tmap_sfa, a.a_sf, ((a.M + 127) / 128) * katoms)) return cudaErrorInvalidValue;
     if (!make_sf_tmap(enc, &tmap_sfw, a.w_sf, ((a.N + 255) / 256) * 2 * katoms)) return cudaErrorInvalidValue;
+    if (!make_y_tmap(enc, &tmap_y, a.Y, a.M, a.N, a.ldy)) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -428,7 +468,7 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     int pairs = sms / 2;
     if (tiles < pairs) pairs = tiles;
     gemm_nvfp4_pair_kernel<<<2 * pairs, kThreads, SMEM_BYTES, stream>>>(
-        tmap_a, tmap_w, tmap_sfa, tmap_sfw, a.hdr, a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy,
+        tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr, a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy,
         (int)a.M, (int)a.N, (int)a.K, a.status, a.probe);
     return cudaGetLastError();
 }
