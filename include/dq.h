@@ -61,8 +61,9 @@ const char *dq_status_string(int status);
 /*
  * Size of the device buffer dq_pack_weights needs for the requested encodings.
  * Storage follows App. A.3 "Storage cost": NVFP4 4.5 bit and LUT3 3.5 bit per
- * weight (codes plus one FP8 scale per 16 weights), plus a 1 KiB header and
- * padding of the NVFP4 scale tiles to 256 rows.
+ * weight (codes plus one FP8 scale per 16 weights), plus a 1 KiB header, a 64 KiB
+ * lookup table for the decode kernel (LUT3 only), padding of the NVFP4 scale tiles to
+ * 256 rows and of LUT3 rows to a multiple of 1024 weights.
  * `formats` must contain at most one of DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3;
  * DQ_FMT_NVFP4_FROM_LUT3 implies DQ_FMT_LUT3.
  */

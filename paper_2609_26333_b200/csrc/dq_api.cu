@@ -157,6 +157,7 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
         }
         if (dq::launch_pack_lut3(W_dev, w_dtype, N, K, ldw, hdr, base + L.lut_off, s) != cudaSuccess)
             return DQ_ERR_CUDA;
+        if (dq::launch_build_lut_table(hdr, base + L.lut_table_off, s) != cudaSuccess) return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
         if (dq::launch_autocast(hdr, base + L.lut_off, N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
@@ -291,6 +292,7 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
     if (st != DQ_OK) return st;
     dq::GemvArgs g;
     g.lut = w->base + w->layout.lut_off;
+    g.table = w->base + w->layout.lut_table_off;
     g.status = status_word_ptr();
     if (!g.status) return DQ_ERR_CUDA;
     g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);

@@ -30,6 +30,7 @@ struct PackedHeader {
     unsigned int autocast_map;    // 8 nibbles: E2M1 code of each level
 };
 constexpr size_t kHeaderBytes = 1024;
+constexpr size_t kLutTableBytes = 65536;   // 256 entries x 32 lane slots x (fp32, fp32): the decode kernel's shared-memory table
 
 // LUT3 device layout: the weights of one row are cut into slices of 1024 (one per warp of the
 // decode kernel); slice s of row r is one block of 448 bytes:
@@ -54,6 +55,7 @@ __host__ __device__ inline size_t lut_scale_offset(int64_t r, int64_t b, int64_t
 struct PackedLayout {
     size_t nv_codes_off = 0, nv_codes_bytes = 0;     // uint8[N][K/2]
     size_t nv_sf_off = 0, nv_sf_bytes = 0;           // [ceil(N/256)*2][K/64][512] MMA scale layout
+    size_t lut_table_off = 0;                        // 64 KiB decode lookup table (level pairs, one slot per lane)
     size_t lut_off = 0, lut_bytes = 0;               // [N][ceil(K/1024)] blocks of kLutBlockBytes (see below)
     size_t total = 0;
 };
@@ -73,6 +75,8 @@ inline PackedLayout packed_layout(int64_t N, int64_t K, unsigned formats)
         off = align_up(off + L.nv_sf_bytes, 1024);
     }
     if (formats & (DQ_FMT_LUT3 | DQ_FMT_NVFP4_FROM_LUT3)) {
+        L.lut_table_off = off;
+        off += kLutTableBytes;
         L.lut_off = off;
         L.lut_bytes = (size_t)N * lut_slices(K) * kLutBlockBytes;
         off = align_up(off + L.lut_bytes, 1024);
@@ -112,6 +116,7 @@ cudaError_t launch_absmax(const void *W, int w_dtype, int64_t N, int64_t K, int6
                           cudaStream_t stream);
 cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
                               const PackedHeader *hdr, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream);
+cudaError_t launch_build_lut_table(const PackedHeader *hdr, uint8_t *table_dev, cudaStream_t stream);
 cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
                              const PackedHeader *hdr, uint8_t *lut_dev, cudaStream_t stream);
 cudaError_t launch_autocast(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
@@ -143,6 +148,7 @@ int gemm_init_driver_api();   // resolves the tensor-map encoder; 0 on success
 
 struct GemvArgs {
     const uint8_t *lut; const PackedHeader *hdr;          // LUT3 blocks (planes + scales)
+    const uint8_t *table = nullptr;                      // prebuilt 64 KiB pair table
     StatusWord *status = nullptr;
     const void *X; int64_t ldx; int64_t B;
     void *Y; int64_t ldy;

@@ -162,7 +162,8 @@ __device__ __forceinline__ void dot32_rows(const uint32_t (&p0)[R], const uint32
 
 template <int BT, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
-gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
+gemv_lut3_kernel(const uint8_t *__restrict__ lut, const uint8_t *__restrict__ table_img,
+                 const PackedHeader *__restrict__ hdr,
                  const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0,
                  int B, __nv_bfloat16 *__restrict__ Y, int64_t ldy, int N, int K, int W, int G, int S,
                  StatusWord *status)
@@ -170,10 +171,9 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict
     extern __shared__ __align__(16) uint8_t smem_raw[];
     const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
     // shared window: [win0, +4 KiB) control | ring part A up to 64 KiB | table 64..128 KiB | ring part B
-    uint8_t *table = smem_raw + (kTableWindowAddr - win0);
     float *red = reinterpret_cast<float *>(smem_raw);                       // [G][2][rows][BT][W] partial sums
-    float *lv = reinterpret_cast<float *>(smem_raw + 2048);                 // 8 codebook levels
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + 2048 + 64);
+    const uint32_t table_bar = win0 + 2048 + 96;                            // arrival of the table image
     const uint32_t bar0 = win0 + 2048 + 128;                                // full[G*S], empty[G*S]
 
     const int lane = threadIdx.x & 31;
@@ -211,6 +211,7 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict
     }
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        tc::mbar_init(table_bar, 1);
         for (int i = 0; i < G * S; ++i) {
             tc::mbar_init(bar0 + 8u * i, 1);                       // full: one producer arrival + bytes
             tc::mbar_init(bar0 + 8u * (G * S + i), (uint32_t)W);   // empty: one arrival per consumer warp
@@ -218,8 +219,12 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (threadIdx.x < 8) lv[threadIdx.x] = hdr->lut_levels[threadIdx.x];
     __syncthreads();
+    // the 64 KiB pair table was built at pack time: one bulk copy brings it in while set-up continues
+    if (threadIdx.x == 0) {
+        tc::mbar_expect_tx(table_bar, kTableBytes);
+        tc::bulk_load(kTableWindowAddr, table_img, kTableBytes, table_bar);
+    }
 
     // producer of this group: lane 0 of its first warp streams whole row blocks into the ring
     const bool producer = (w == 0 && lane == 0);
@@ -232,14 +237,6 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict
                 tc::bulk_load(chunk_addr(s), lut + (size_t)rb * chunk_bytes, chunk_bytes, full_bar(s));
             }
         }
-    }
-
-    // level-pair table: entry e (a byte of merged plane bits) -> (G[idx_a], G[idx_b]) as fp32, one slot per lane
-    for (int i = threadIdx.x; i < 256 * 32; i += blockDim.x) {
-        const int e = i >> 5, l = i & 31;
-        const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
-        const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
-        *reinterpret_cast<float2 *>(table + e * 256 + l * 8) = make_float2(lv[ia], lv[ib]);
     }
 
     // this lane's 32 activations per batch column, widened to fp32 pairs, kept in registers
@@ -258,11 +255,15 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict
         }
     }
     const float s_w = hdr->s;
-    __syncthreads();
+    bool ok = true;
+    {   // table image must have landed before the first lookup
+        uint32_t good = 1;
+        if (lane == 0) good = gemv_wait(table_bar, 0u, abort_flag) ? 1u : 0u;
+        ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+    }
 
     int it = 0, stage = 0;
     uint32_t phase = 0;
-    bool ok = true;
     const uint32_t lane_off = (uint32_t)w * kLutBlockBytes + (uint32_t)lane * 4;
     const uint32_t sc_off = (uint32_t)w * kLutBlockBytes + kLutScaleOff + (uint32_t)lane * 2;
     for (int rb = first; rb < nblocks; rb += stride, ++it) {
@@ -368,7 +369,7 @@ static cudaError_t launch_one(const GemvArgs &a, int b0, int grid, int threads, 
         attr_set = true;
     }
     gemv_lut3_kernel<BT, MAXT><<<grid, threads, kDynSmemBytes, stream>>>(
-        a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X), a.ldx, b0, (int)a.B,
+        a.lut, a.table, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X), a.ldx, b0, (int)a.B,
         reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy, (int)a.N, (int)a.K, W, G, S, a.status);
     return cudaGetLastError();
 }

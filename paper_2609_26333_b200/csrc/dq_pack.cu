@@ -193,6 +193,27 @@ cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, 
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------- decode pair table
+
+// Image of the decode kernel's shared-memory table, built once at pack time: entry e (a byte holding
+// the index bits b0a b0b b1a b1b b2a b2b of two neighbouring weights) -> (G[idx_a], G[idx_b]) as fp32,
+// replicated into one 8-byte slot per lane (entry stride 256 bytes).
+__global__ void build_lut_table_kernel(const PackedHeader *hdr, uint8_t *table)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 256 * 32) return;
+    const int e = i >> 5, l = i & 31;
+    const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
+    const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
+    *reinterpret_cast<float2 *>(table + e * 256 + l * 8) = make_float2(hdr->lut_levels[ia], hdr->lut_levels[ib]);
+}
+
+cudaError_t launch_build_lut_table(const PackedHeader *hdr, uint8_t *table_dev, cudaStream_t stream)
+{
+    build_lut_table_kernel<<<32, 256, 0, stream>>>(hdr, table_dev);
+    return cudaGetLastError();
+}
+
 // --------------------------------------------------------------- LUT3 pack
 
 // One thread quantises 32 consecutive weights (two 16-blocks) and emits one word of each bit-plane.
@@ -355,6 +376,51 @@ cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, 
 
 // --------------------------------------------------- activation quantiser
 
+// eight floats -> four bytes of E2M1 codes (element 0 in the low nibble of byte 0)
+__device__ __forceinline__ uint32_t f32x8_to_e2m1x8(float f0, float f1, float f2, float f3, float f4, float f5, float f6,
+                                                    float f7)
+{
+    uint32_t r;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(r) : "f"(f0), "f"(f1), "f"(f2), "f"(f3), "f"(f4), "f"(f5), "f"(f6), "f"(f7));
+    return r;
+}
+
+// NVFP4 round-to-nearest of one 16-block held as eight packed bf16 pairs; same arithmetic as
+// quant_block_nvfp4 (the block maximum is exact in bf16, so taking it on packed pairs changes nothing)
+__device__ __forceinline__ uint32_t quant_block_nvfp4_bf16(const uint32_t (&w)[8], float s, float rc6, uint2 &codes)
+{
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t a;
+        asm("abs.bf16x2 %0, %1;" : "=r"(a) : "r"(w[i]));
+        if (i == 0) m = a;
+        else asm("max.bf16x2 %0, %0, %1;" : "+r"(m) : "r"(a));
+    }
+    const float a = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+    const float t = __fmul_rn(a, rc6);
+    const uint32_t d8 = f32_to_e4m3(t);
+    codes = make_uint2(0u, 0u);
+    if ((d8 & 0x7Fu) != 0u) {
+        const float r = __frcp_rn(__fmul_rn(s, e4m3_to_f32(d8)));
+        float y[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            y[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), r);
+            y[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), r);
+        }
+        codes.x = f32x8_to_e2m1x8(y[0], y[1], y[2], y[3], y[4], y[5], y[6], y[7]);
+        codes.y = f32x8_to_e2m1x8(y[8], y[9], y[10], y[11], y[12], y[13], y[14], y[15]);
+    }
+    return d8;
+}
+
 // bf16 -> NVFP4 with a static tensor scale (App. A.3 "NVFP4").  One thread per
 // 16-block: 32 B in, 8 B of codes out; four neighbouring lanes (one 64-wide k
 // atom) merge their scale bytes into one 32-bit store of the MMA scale layout.
@@ -369,10 +435,11 @@ __global__ void __launch_bounds__(256) quant_act_kernel(const __nv_bfloat16 *A, 
     const float rc6 = __frcp_rn(__fmul_rn(6.0f, s));
     uint32_t d8 = 0;
     if (live) {
-        float x[16];
-        load16<false>(A, r, b * 16, lda, x);
+        const uint4 *p = reinterpret_cast<const uint4 *>(A + r * lda + b * 16);
+        const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         uint2 c;
-        d8 = quant_block_nvfp4(x, s, rc6, c);
+        d8 = quant_block_nvfp4_bf16(w, s, rc6, c);
         *reinterpret_cast<uint2 *>(codes + r * (K / 2) + b * 8) = c;
     }
     // K % 64 == 0, so lanes 4q..4q+3 always hold the four blocks of one k atom of one row

@@ -34,11 +34,11 @@ def test_library_exports_every_declared_symbol(dq):
 def test_packed_bytes_follows_storage_cost(dq):
     N, K = 6144, 4096
     nv = dq.packed_bytes(N, K, dq.FMT_NVFP4) - 1024
-    lut = dq.packed_bytes(N, K, dq.FMT_LUT3) - 1024
+    lut = dq.packed_bytes(N, K, dq.FMT_LUT3) - 1024 - 65536      # header + the decode kernel's 64 KiB lookup table
     assert nv == N * K // 2 + N * K // 16           # 4.5 bit per weight
     assert lut == 3 * N * K // 8 + N * K // 16      # 3.5 bit per weight
-    assert dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3) == 1024 + nv + lut
-    assert dq.packed_bytes(N, K, dq.FMT_NVFP4_FROM_LUT3) == 1024 + nv + lut
+    assert dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3) == 1024 + 65536 + nv + lut
+    assert dq.packed_bytes(N, K, dq.FMT_NVFP4_FROM_LUT3) == 1024 + 65536 + nv + lut
 
 
 def test_argument_validation_needs_no_device(dq):
