@@ -48,6 +48,16 @@ C4_LAYERS = 64
 C4_MATRICES = (("q", 8192, 5120), ("k", 1024, 5120), ("v", 1024, 5120), ("o", 5120, 8192),
                ("gate", 17408, 5120), ("up", 17408, 5120), ("down", 5120, 17408))
 C4_PREFILL_M = 4096
+C4_DECODE_BATCHES = (1, 2, 4, 8, 16, 32, 64)
+
+
+def c4_fused_layer(layer: int = 0):
+    """The four matrices one layer of the 27B-class stack serves: q/k/v and gate/up are stored
+    fused (each fused tensor has one global scale), o and down on their own."""
+    shapes = (("qkv", 8192 + 1024 + 1024, 5120), ("o", 5120, 8192), ("gate_up", 2 * 17408, 5120),
+              ("down", 5120, 17408))
+    return [LayerConfig(f"c4_l{layer}_{nm}", N=n, K=k, M=C4_PREFILL_M, decode_batches=C4_DECODE_BATCHES, cfg_id=4,
+                        matrix_id=i) for i, (nm, n, k) in enumerate(shapes)]
 
 
 def seed_of(cfg: LayerConfig, layer: int = 0) -> int:

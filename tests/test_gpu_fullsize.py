@@ -26,11 +26,12 @@ def _f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def _run_config(dq, oracle, name, full_rows):
-    cfg = dq_inputs.CONFIGS[name]
-    W = dq_inputs.make_weight(cfg)
-    A = dq_inputs.make_activations(cfg, cfg.M)
-    X = dq_inputs.make_activations(cfg, max(cfg.decode_batches), salt=2)
+def _run_config(dq, oracle, name, full_rows, layer=0):
+    cfg = name if isinstance(name, dq_inputs.LayerConfig) else dq_inputs.CONFIGS[name]
+    name = cfg.name
+    W = dq_inputs.make_weight(cfg, layer)
+    A = dq_inputs.make_activations(cfg, cfg.M, layer=layer)
+    X = dq_inputs.make_activations(cfg, max(cfg.decode_batches), salt=2, layer=layer)
     sa = dq_inputs.static_act_scale(A)
     w = dq.pack_weights(W.to(DEV))
     ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w, cfg.M), DEV)
@@ -76,3 +77,16 @@ def test_c3_gate_up_sampled(dq, oracle):
 
 def test_c3_down_sampled(dq, oracle):
     _run_config(dq, oracle, "c3_down27b", full_rows=False)
+
+
+def test_c5_outlier_sampled(dq, oracle):
+    """70B-class layer with heavy-tailed activations and x50 outlier channels under a static
+    activation scale: block scales saturate and underflow on both sides in the same way."""
+    _run_config(dq, oracle, "c5_outlier70b", full_rows=False)
+
+
+@pytest.mark.parametrize("which", [0, 1, 2, 3])
+def test_c4_stack_layer_shapes(dq, oracle, which):
+    """The matrices of one layer of the 27B-class stack (fused q/k/v, o, fused gate/up, down) at
+    4096 prefill tokens and decode batches 1..64; the other 63 layers repeat these shapes."""
+    _run_config(dq, oracle, dq_inputs.c4_fused_layer(layer=3)[which], full_rows=False, layer=3)

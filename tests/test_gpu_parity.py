@@ -264,3 +264,37 @@ def test_calls_reject_wrong_handle_use(dq, oracle):
     with pytest.raises(dq.DQError):
         dq.prefill_linear(w_nv, A, -1.0)
     _status_ok(dq)
+
+
+def test_calls_replay_from_a_cuda_graph(dq, oracle):
+    """Prefill and decode calls neither allocate nor synchronise, so a stream capture records
+    them; replays on new inputs (same buffers) give what eager calls give, bit for bit."""
+    M, N, K = 384, 512, 1024
+    W, ref = _layer(oracle, N, K, 70)
+    w = dq.pack_weights(W.to(DEV))
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w, M), DEV)
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, 71).to(DEV)
+    X = dq_inputs.gaussian_bf16(4, K, 1.0, 72).to(DEV)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    Yd = torch.empty(4, N, dtype=torch.bfloat16, device=DEV)
+    sa = 4.0 / 2688.0
+    dq.prefill_linear(w, A, sa, out=Y, workspace=ws)     # first calls outside capture (one-time set-up)
+    dq.decode_linear(w, X, out=Yd)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        dq.prefill_linear(w, A, sa, out=Y, workspace=ws)
+        dq.decode_linear(w, X, out=Yd)
+    for seed in (73, 74):
+        A.copy_(dq_inputs.gaussian_bf16(M, K, 1.0, seed).to(DEV))
+        X.copy_(dq_inputs.gaussian_bf16(4, K, 1.0, seed + 10).to(DEV))
+        Y.zero_(); Yd.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got, got_d = Y.clone(), Yd.clone()
+        want = dq.prefill_linear(w, A, sa, workspace=ws)
+        want_d = dq.decode_linear(w, X)
+        _status_ok(dq)
+        assert torch.equal(got, want) and torch.equal(got_d, want_d)
+    Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A.cpu()), sa, ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, "graph replay prefill")
