@@ -97,7 +97,8 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
 /* Frees the host handle only; the packed device buffer belongs to the caller. */
 int dq_free_weights(dq_weights *w);
 
-/* Scratch dq_prefill_linear needs for M tokens (NVFP4 activation codes + scales). */
+/* Scratch dq_prefill_linear needs for M tokens: NVFP4 activation codes + scales, and for a
+ * handle packed with DQ_FMT_LUT3 only also the NVFP4 view of the weights (see below). */
 int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_host);
 
 /*
@@ -107,6 +108,12 @@ int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_hos
  * scale `act_global_scale` (App. A.3 "NVFP4": s_a in  a^ = s_a * d_b * e2m1) and
  * W^ the handle's NVFP4 weights; block-scaled FP4 tensor-core GEMM, fp32
  * accumulation.
+ * A handle packed with DQ_FMT_LUT3 alone stores one 3.5-bit matrix for both phases
+ * (Sec. 2.3 "format-disaggregated LUT3"; the paper describes this on-the-fly cast but
+ * does not build it): every prefill call first casts the LUT3 codes to NVFP4 into the
+ * workspace (integer code map, block scale |d_b|, same tensor scale; the result equals
+ * the DQ_FMT_NVFP4_FROM_LUT3 view bit for bit) and then runs the same GEMM.  The cast
+ * is part of dq_prefill_quantize when the two stages are called separately.
  * A_dev: M x K bf16, row stride lda; Y_dev: M x N bf16, row stride ldy.
  * act_global_scale must be finite and > 0.  M >= 1.
  * workspace_dev: at least dq_prefill_workspace_bytes(M) bytes, private to this

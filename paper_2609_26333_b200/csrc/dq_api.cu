@@ -54,6 +54,25 @@ int check_formats(unsigned formats)
 
 bool valid_handle(const dq_weights *w) { return w != nullptr && w->magic == kMagic; }
 
+// Prefill workspace: NVFP4 activations (codes, MMA-layout scales); for a handle that stores only
+// LUT3 the NVFP4 view of the weights (codes, MMA-layout scales) follows, rebuilt on every call.
+struct WsLayout { size_t a_sf = 0, w_codes = 0, w_sf = 0, w_sf_bytes = 0, total = 0; };
+bool has_nvfp4_view(const dq_weights *w) { return (w->formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3)) != 0; }
+WsLayout ws_layout(const dq_weights *w, int64_t M)
+{
+    WsLayout L;
+    L.a_sf = dq::align_up((size_t)M * w->K / 2, 1024);
+    const size_t sf = dq::align_up((size_t)M, dq::kSfAtomRows) * (size_t)(w->K / dq::kBlock);
+    L.total = L.a_sf + dq::align_up(sf, 1024);
+    if (!has_nvfp4_view(w)) {
+        L.w_codes = L.total;
+        L.w_sf = L.w_codes + dq::align_up((size_t)w->N * w->K / 2, 1024);
+        L.w_sf_bytes = dq::align_up((size_t)w->N, dq::kSfRowPad) * (size_t)(w->K / dq::kBlock);
+        L.total = L.w_sf + dq::align_up(L.w_sf_bytes, 1024);
+    }
+    return L;
+}
+
 dq::StatusWord *status_word_ptr()
 {
     void *p = nullptr;
@@ -197,9 +216,7 @@ int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsi
 int dq_prefill_workspace_bytes(const dq_weights *w, int64_t M, size_t *bytes_host)
 {
     if (!valid_handle(w) || !bytes_host || M < 1) return DQ_ERR_INVALID_ARG;
-    const size_t codes = dq::align_up((size_t)M * w->K / 2, 1024);
-    const size_t sf = dq::align_up((size_t)M, dq::kSfAtomRows) * (size_t)(w->K / dq::kBlock);
-    *bytes_host = codes + dq::align_up(sf, 1024);
+    *bytes_host = ws_layout(w, M).total;
     return DQ_OK;
 }
 
@@ -207,7 +224,7 @@ static int prefill_checks(const dq_weights *w, int64_t M, float act_global_scale
                           size_t workspace_bytes)
 {
     if (!valid_handle(w) || !workspace_dev) return DQ_ERR_INVALID_ARG;
-    if (!(w->formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3))) return DQ_ERR_INVALID_ARG;
+    if (!has_nvfp4_view(w) && !(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
     if (M < 1 || M > (1ll << 24)) return DQ_ERR_INVALID_ARG;
     if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
     if (!aligned(workspace_dev, 1024)) return DQ_ERR_ALIGN;
@@ -227,10 +244,19 @@ int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64
     st = check_arch();
     if (st != DQ_OK) return st;
     uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
-    uint8_t *a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
-    if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, ws, a_sf, 1,
-                             reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    const WsLayout L = ws_layout(w, M);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, ws, ws + L.a_sf, 1, s) != cudaSuccess)
         return DQ_ERR_CUDA;
+    if (!has_nvfp4_view(w)) {
+        // the stored matrix is LUT3 only: cast it to NVFP4 for this call (Sec. 2.3, same code map as the
+        // pack-time view); rows that pad the scale layout to the GEMM tile must read as zero
+        if (w->N % dq::kSfRowPad != 0 && cudaMemsetAsync(ws + L.w_sf, 0, L.w_sf_bytes, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+        if (dq::launch_autocast(reinterpret_cast<const dq::PackedHeader *>(w->base), w->base + w->layout.lut_off, w->N,
+                                w->K, ws + L.w_codes, ws + L.w_sf, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
     return DQ_OK;
 }
 
@@ -250,10 +276,11 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
     if (!sw) return DQ_ERR_CUDA;
     const uint8_t *ws = reinterpret_cast<const uint8_t *>(workspace_dev);
     dq::GemmArgs g;
+    const WsLayout L = ws_layout(w, M);
     g.a_codes = ws;
-    g.a_sf = ws + dq::align_up((size_t)M * w->K / 2, 1024);
-    g.w_codes = w->base + w->layout.nv_codes_off;
-    g.w_sf = w->base + w->layout.nv_sf_off;
+    g.a_sf = ws + L.a_sf;
+    g.w_codes = has_nvfp4_view(w) ? w->base + w->layout.nv_codes_off : ws + L.w_codes;
+    g.w_sf = has_nvfp4_view(w) ? w->base + w->layout.nv_sf_off : ws + L.w_sf;
     g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
     g.act_scale = act_global_scale;
     g.Y = Y_dev;

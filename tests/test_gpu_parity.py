@@ -200,6 +200,34 @@ def test_prefill_strided_output_and_autocast_weights(dq, oracle):
     check_outputs(_f64(out[:, :N]), Yr, S, "prefill on autocast weights")
 
 
+def test_prefill_on_lut3_only_handle_casts_at_call_time(dq, oracle):
+    """One stored 3.5-bit matrix serves both phases: the prefill call casts LUT3 to NVFP4 into
+    its workspace.  Same result, bit for bit, as the pack-time view; parity against the oracle's
+    autocast codes; N is not a multiple of the GEMM tile so the scale padding path runs."""
+    M, N, K = 300, 784, 1152
+    W, ref = _layer(oracle, N, K, 32)
+    Wd = W.to(DEV)
+    w_lut = dq.pack_weights(Wd, formats=dq.FMT_LUT3)
+    w_view = dq.pack_weights(Wd, formats=dq.FMT_NVFP4_FROM_LUT3)
+    assert dq.packed_bytes(N, K, dq.FMT_LUT3) < dq.packed_bytes(N, K, dq.FMT_NVFP4_FROM_LUT3)
+    assert dq.prefill_workspace_bytes(w_lut, M) > dq.prefill_workspace_bytes(w_view, M)
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, 55)
+    sa = dq_inputs.static_act_scale(A)
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w_lut, M), DEV)
+    ws.fill_(0xFF)                                   # stale workspace contents must not matter
+    Y1 = dq.prefill_linear(w_lut, A.to(DEV), sa, workspace=ws)
+    Y1b = dq.prefill_linear(w_lut, A.to(DEV), sa, workspace=ws)
+    Y2 = dq.prefill_linear(w_view, A.to(DEV), sa)
+    _status_ok(dq)
+    assert torch.equal(Y1, Y2) and torch.equal(Y1, Y1b)
+    ac = oracle.autocast_lut3_to_nvfp4(ref["lut3_planes"], ref["lut3_scales"])
+    Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa, ac[0], ac[1], ref["s"])
+    check_outputs(_f64(Y1), Yr, S, "prefill on a LUT3-only handle")
+    y = dq.decode_linear(w_lut, A[:2].to(DEV))       # and the same handle still decodes
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(A[:2]), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    check_outputs(_f64(y), Yr, S, "decode on the same handle")
+
+
 def test_prefill_outlier_activations(dq, oracle):
     M, N, K = 256, 512, 1024
     W, ref = _layer(oracle, N, K, 57)
@@ -252,9 +280,6 @@ def test_calls_reject_wrong_handle_use(dq, oracle):
     w_lut = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
     w_nv = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
     A = dq_inputs.gaussian_bf16(4, K, 1.0, 66).to(DEV)
-    with pytest.raises(dq.DQError) as e:
-        dq.prefill_linear(w_lut, A, 1.0)
-    assert e.value.code == 1
     with pytest.raises(dq.DQError) as e:
         dq.decode_linear(w_nv, A)
     assert e.value.code == 1
