@@ -135,7 +135,8 @@ def run_reference(args, cfg):
         return
     import oracle
     oracle.build()
-    rows = args.ref_rows
+    # rows per step: about 0.9 s of oracle work, so that the default 200 steps end within minutes
+    rows = args.ref_rows or max(16, min(cfg.M, int(0.9 * 0.05e12 / (2.0 * cfg.N * cfg.K)) // 16 * 16))
     W = dq_inputs.make_weight(cfg)
     W_f32 = dq_inputs.bf16_to_f32_numpy(W)
     A = dq_inputs.make_activations(cfg, rows)
@@ -178,7 +179,8 @@ def main():
     ap.add_argument("--impl", default="dq", choices=["dq", "reference"])
     ap.add_argument("--decode-batch", type=int, default=1)
     ap.add_argument("--copies", type=int, default=0, help="rotating packed-weight copies (0 = enough to exceed 2x L2)")
-    ap.add_argument("--ref-rows", type=int, default=128, help="prefill rows per oracle step")
+    ap.add_argument("--ref-rows", type=int, default=0,
+                    help="prefill rows per oracle pass (0 = 2048 for cpu_baseline; sized to a ~3 minute run for --impl reference)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -319,16 +321,14 @@ def main():
         e2e = {"prefill_ms": p_ms, "decode_ms": dd_ms, "steps": n_e2e}
 
     # ---- max over ranks ----
-    times = torch.tensor([total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0,
-                          e2e["decode_ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms = [float(v) for v in times.cpu()]
+    from paper_2609_26333_b200 import replicas
+    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms = replicas.max_over_ranks(
+        [total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0, e2e["decode_ms"] if e2e else 0.0], device=dev)
 
     flops = 2.0 * M * N * K
     dec_bytes = 0.4375 * N * K + 2.0 * B * K + 2.0 * B * N + 4
     quant_bytes = 2.5625 * M * K
-    prefill_tflops = world * flops / ((q_ms + g_ms) * 1e-3) / 1e12
+    prefill_tflops = replicas.whole_job_rate(flops, world, q_ms + g_ms) / 1e12
     gemm_tflops = flops / (g_ms * 1e-3) / 1e12
     decode_gbs = dec_bytes / (d_ms * 1e-3) / 1e9
     quant_gbs = quant_bytes / (q_ms * 1e-3) / 1e9
@@ -369,7 +369,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         oracle.build()
-        rows = args.ref_rows
+        rows = min(M, args.ref_rows or 2048)
         W_f32 = dq_inputs.bf16_to_f32_numpy(dq_inputs.make_weight(cfg))
         A_f32 = dq_inputs.bf16_to_f32_numpy(A_host[:rows])
         X_f32 = dq_inputs.bf16_to_f32_numpy(X_host)

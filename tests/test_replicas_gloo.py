@@ -1,0 +1,53 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks, max over ranks of the per-rank times and
+the whole-job rate derived from it."""
+import os
+import socket
+import sys
+
+import pytest
+import torch
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2609_26333_b200 import replicas
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        dist.barrier()
+        mine = [10.0 + rank, 5.0 - rank, 0.25 * (rank + 1)]          # per-rank device times (ms)
+        got = replicas.max_over_ranks(mine)
+        rate = replicas.whole_job_rate(units_per_rank=1.0e12, world=world, slowest_ms=got[0])
+        dist.barrier()
+        torch.save({"got": got, "rate": rate}, os.path.join(out_dir, f"r{rank}.pt"))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_max_and_whole_job_rate(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    for rank in range(world):
+        r = torch.load(os.path.join(str(tmp_path), f"r{rank}.pt"))
+        assert r["got"] == [11.0, 5.0, 0.5]                           # same on every rank
+        assert r["rate"] == pytest.approx(2 * 1.0e12 / 11.0e-3)
+
+
+def test_single_process_is_identity():
+    sys.path.insert(0, ROOT)
+    from paper_2609_26333_b200 import replicas
+
+    assert replicas.max_over_ranks([3.0, 1.5]) == [3.0, 1.5]
+    assert replicas.whole_job_rate(2.0, 1, 1000.0) == 2.0
