@@ -185,6 +185,20 @@ int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, v
                         float *global_scale_dev, void *stream);
 
 /*
+ * The inverse: build a handle from canonical encodings (layouts as above, device pointers), e.g.
+ * weights quantised elsewhere with the same formats (App. A.3).  `formats` as in dq_pack_weights:
+ * DQ_FMT_NVFP4 needs nvfp4_codes_dev / nvfp4_scales_dev, DQ_FMT_LUT3 and DQ_FMT_NVFP4_FROM_LUT3
+ * need lut3_planes_dev / lut3_scales_dev (unused pointers may be NULL); global_scale is the tensor
+ * scale s (finite, > 0), shared by both encodings.  packed_dev / packed_bytes / ownership as in
+ * dq_pack_weights.  No value check is made on the codes: every bit pattern decodes to something.
+ */
+int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp4_codes_dev,
+                        const void *nvfp4_scales_dev, const void *lut3_planes_dev,
+                        const void *lut3_scales_dev, float global_scale,
+                        const uint16_t *lut3_codebook_f16_host, void *packed_dev, size_t packed_bytes,
+                        void *stream, dq_weights **out_host);
+
+/*
  * The activation quantiser of dq_prefill_linear on its own (App. A.3 "NVFP4",
  * static input scale), writing canonical layout:
  *   codes uint8[M][K/2], scales uint8[M][K/16].

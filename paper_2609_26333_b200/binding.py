@@ -20,7 +20,7 @@ DT_FP32 = 1
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
-           "dq_decode_linear", "dq_export_canonical",
+           "dq_decode_linear", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
 
 
@@ -65,6 +65,9 @@ def lib() -> C.CDLL:
         L.dq_prefill_linear_static.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp]
         L.dq_decode_linear.restype = C.c_int
         L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_import_canonical.restype = C.c_int
+        L.dq_import_canonical.argtypes = [C.c_int64, C.c_int64, C.c_uint, vp, vp, vp, vp, C.c_float,
+                                          C.POINTER(C.c_uint16), vp, C.c_size_t, vp, C.POINTER(vp)]
         L.dq_export_canonical.restype = C.c_int
         L.dq_export_canonical.argtypes = [vp, C.c_uint, vp, vp, vp, vp]
         L.dq_quantize_activations.restype = C.c_int
@@ -141,6 +144,31 @@ def pack_weights(W: torch.Tensor, formats: int = FMT_NVFP4 | FMT_LUT3, codebook_
     out = C.c_void_p(0)
     _check(lib().dq_pack_weights(W.data_ptr(), dt, N, K, W.stride(0), formats, cb, view.data_ptr(), nbytes,
                                  _stream_ptr(stream), C.byref(out)), "dq_pack_weights")
+    if formats & FMT_NVFP4_FROM_LUT3:
+        formats |= FMT_LUT3
+    return DQWeights(out.value, packed, N, K, formats)
+
+
+def import_canonical(N: int, K: int, formats: int, global_scale: float, nvfp4=None, lut3=None, codebook_f16=None,
+                     stream=None) -> DQWeights:
+    """dq_import_canonical: handle from canonical (codes, scales) pairs of CUDA tensors."""
+    dev = (nvfp4 or lut3)[0].device
+    nbytes = packed_bytes(N, K, formats)
+    packed = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+    off = (-packed.data_ptr()) % 1024
+    view = packed[off:off + nbytes]
+    cb = None
+    if codebook_f16 is not None:
+        cb = (C.c_uint16 * 8)(*[int(v) for v in codebook_f16])
+    ptr = lambda pair, i: pair[i].data_ptr() if pair is not None else None
+    if nvfp4 is not None:
+        assert nvfp4[0].is_contiguous() and nvfp4[1].is_contiguous() and nvfp4[0].shape == (N, K // 2)
+    if lut3 is not None:
+        assert lut3[0].is_contiguous() and lut3[1].is_contiguous() and lut3[0].shape == (N, 3, K // 32)
+    out = C.c_void_p(0)
+    _check(lib().dq_import_canonical(N, K, formats, ptr(nvfp4, 0), ptr(nvfp4, 1), ptr(lut3, 0), ptr(lut3, 1),
+                                     float(global_scale), cb, view.data_ptr(), nbytes, _stream_ptr(stream),
+                                     C.byref(out)), "dq_import_canonical")
     if formats & FMT_NVFP4_FROM_LUT3:
         formats |= FMT_LUT3
     return DQWeights(out.value, packed, N, K, formats)

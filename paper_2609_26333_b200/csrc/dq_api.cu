@@ -196,6 +196,72 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
     return DQ_OK;
 }
 
+int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp4_codes_dev,
+                        const void *nvfp4_scales_dev, const void *lut3_planes_dev, const void *lut3_scales_dev,
+                        float global_scale, const uint16_t *lut3_codebook_f16_host, void *packed_dev,
+                        size_t packed_bytes, void *stream, dq_weights **out_host)
+{
+    if (!packed_dev || !out_host) return DQ_ERR_INVALID_ARG;
+    int st = check_formats(formats);
+    if (st != DQ_OK) return st;
+    st = check_shape(N, K);
+    if (st != DQ_OK) return st;
+    if (!(global_scale > 0.0f) || !std::isfinite(global_scale)) return DQ_ERR_INVALID_ARG;
+    if (formats & DQ_FMT_NVFP4_FROM_LUT3) formats |= DQ_FMT_LUT3;
+    if ((formats & DQ_FMT_NVFP4) && (!nvfp4_codes_dev || !nvfp4_scales_dev)) return DQ_ERR_INVALID_ARG;
+    if ((formats & DQ_FMT_LUT3) && (!lut3_planes_dev || !lut3_scales_dev)) return DQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 1024)) return DQ_ERR_ALIGN;
+    if ((formats & DQ_FMT_NVFP4) && (!aligned(nvfp4_codes_dev, 8))) return DQ_ERR_ALIGN;
+    if ((formats & DQ_FMT_LUT3) && (!aligned(lut3_planes_dev, 4))) return DQ_ERR_ALIGN;
+    uint16_t cb[8];
+    if (lut3_codebook_f16_host) std::memcpy(cb, lut3_codebook_f16_host, sizeof(cb));
+    else default_codebook(cb);
+    if (!valid_codebook(cb)) return DQ_ERR_INVALID_ARG;
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    const dq::PackedLayout L = dq::packed_layout(N, K, formats);
+    if (packed_bytes < L.total) return DQ_ERR_WORKSPACE;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint8_t *base = reinterpret_cast<uint8_t *>(packed_dev);
+    dq::PackedHeader *hdr = reinterpret_cast<dq::PackedHeader *>(base);
+    if (cudaMemsetAsync(base, 0, dq::kHeaderBytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_pack_header(hdr, cb, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_set_scale(hdr, global_scale, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (L.nv_sf_bytes && cudaMemsetAsync(base + L.nv_sf_off, 0, L.nv_sf_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (formats & DQ_FMT_NVFP4) {
+        if (dq::launch_import_nvfp4(reinterpret_cast<const uint8_t *>(nvfp4_codes_dev),
+                                    reinterpret_cast<const uint8_t *>(nvfp4_scales_dev), N, K, base + L.nv_codes_off,
+                                    base + L.nv_sf_off, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_LUT3) {
+        if (L.lut_bytes != (size_t)N * K / 16 * 7 && cudaMemsetAsync(base + L.lut_off, 0, L.lut_bytes, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
+        if (dq::launch_import_lut3(reinterpret_cast<const uint32_t *>(lut3_planes_dev),
+                                   reinterpret_cast<const uint8_t *>(lut3_scales_dev), N, K, base + L.lut_off, s) !=
+            cudaSuccess)
+            return DQ_ERR_CUDA;
+        if (dq::launch_build_lut_table(hdr, base + L.lut_table_off, s) != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
+        if (dq::launch_autocast(hdr, base + L.lut_off, N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
+            cudaSuccess)
+            return DQ_ERR_CUDA;
+    }
+    dq_weights *w = new (std::nothrow) dq_weights;
+    if (!w) return DQ_ERR_INTERNAL;
+    w->magic = kMagic;
+    cudaGetDevice(&w->device);
+    w->N = N;
+    w->K = K;
+    w->formats = formats;
+    w->base = base;
+    w->layout = L;
+    *out_host = w;
+    return DQ_OK;
+}
+
 int dq_free_weights(dq_weights *w)
 {
     if (!valid_handle(w)) return DQ_ERR_INVALID_ARG;

@@ -127,6 +127,11 @@ cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, c
 cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                                int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
                                cudaStream_t stream);
+cudaError_t launch_set_scale(PackedHeader *hdr, float s, cudaStream_t stream);
+cudaError_t launch_import_nvfp4(const uint8_t *codes_in, const uint8_t *scales_in, int64_t N, int64_t K, uint8_t *codes,
+                                uint8_t *sf_swizzled, cudaStream_t stream);
+cudaError_t launch_import_lut3(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                               uint8_t *lut_dev, cudaStream_t stream);
 // Activation quantiser: codes row-major [M][K/2]; scales either in the MMA layout
 // (swizzled != 0) or canonical [M][K/16].
 cudaError_t launch_quant_act(const void *A_bf16, int64_t M, int64_t K, int64_t lda, float act_scale, uint8_t *codes,

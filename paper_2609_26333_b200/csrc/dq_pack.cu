@@ -374,6 +374,71 @@ cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, 
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ import
+
+// Canonical codes / scales (the layouts of the export) -> device layouts.  Inverse of the export kernels.
+__global__ void import_nvfp4_kernel(const uint8_t *codes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                                    uint8_t *codes, uint8_t *sf)
+{
+    const int64_t nb = K / 16;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * nb) return;
+    const int64_t r = i / nb, b = i % nb;
+    *reinterpret_cast<uint2 *>(codes + r * (K / 2) + b * 8) =
+        *reinterpret_cast<const uint2 *>(codes_in + r * (K / 2) + b * 8);
+    sf[sf_swizzled_offset(r, b, K)] = scales_in[r * nb + b];
+}
+
+__global__ void import_lut3_kernel(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                                   uint8_t *lut)
+{
+    const int64_t nw = K / 32;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * nw) return;
+    const int64_t r = i / nw, j = i % nw;
+#pragma unroll
+    for (int p = 0; p < 3; ++p) {
+        const uint32_t c = planes_in[(r * 3 + p) * nw + j];                        // canonical: LSB-first
+        uint32_t w = 0;
+#pragma unroll
+        for (int b = 0; b < 32; ++b) w |= ((c >> b) & 1u) << lut3_bitpos(p, b);
+        *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = w;
+    }
+    lut[lut_scale_offset(r, 2 * j, K)] = scales_in[r * (K / 16) + 2 * j];
+    lut[lut_scale_offset(r, 2 * j + 1, K)] = scales_in[r * (K / 16) + 2 * j + 1];
+}
+
+__global__ void set_scale_kernel(PackedHeader *hdr, float s)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    hdr->s = s;
+    hdr->rc6 = __frcp_rn(__fmul_rn(6.0f, s));
+    hdr->amax_bits = __float_as_uint(__fmul_rn(s, 2688.0f));
+}
+
+cudaError_t launch_set_scale(PackedHeader *hdr, float s, cudaStream_t stream)
+{
+    set_scale_kernel<<<1, 32, 0, stream>>>(hdr, s);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_import_nvfp4(const uint8_t *codes_in, const uint8_t *scales_in, int64_t N, int64_t K, uint8_t *codes,
+                                uint8_t *sf_swizzled, cudaStream_t stream)
+{
+    const int64_t total = N * (K / 16);
+    import_nvfp4_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(codes_in, scales_in, N, K, codes,
+                                                                             sf_swizzled);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_import_lut3(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                               uint8_t *lut_dev, cudaStream_t stream)
+{
+    const int64_t total = N * (K / 32);
+    import_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(planes_in, scales_in, N, K, lut_dev);
+    return cudaGetLastError();
+}
+
 // --------------------------------------------------- activation quantiser
 
 // eight floats -> four bytes of E2M1 codes (element 0 in the low nibble of byte 0)

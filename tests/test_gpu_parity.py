@@ -125,6 +125,34 @@ def test_autocast_view_bit_exact(dq, oracle):
     assert np.array_equal(_np(codes), ac) and np.array_equal(_np(scales), asc)
 
 
+def test_import_canonical_round_trip_and_use(dq, oracle):
+    """Oracle-made codes go in through dq_import_canonical, come back unchanged through the export,
+    and drive both kernels to the same results as a handle packed from the master weights."""
+    M, N, K = 160, 272, 640
+    W, ref = _layer(oracle, N, K, 36)
+    nv = (torch.from_numpy(ref["nvfp4_codes"]).to(DEV), torch.from_numpy(ref["nvfp4_scales"]).to(DEV))
+    lut = (torch.from_numpy(ref["lut3_planes"].view(np.int32)).to(DEV), torch.from_numpy(ref["lut3_scales"]).to(DEV))
+    w_imp = dq.import_canonical(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3, float(ref["s"]), nvfp4=nv, lut3=lut)
+    w_pack = dq.pack_weights(W.to(DEV))
+    for fmt, want in ((dq.FMT_NVFP4, (ref["nvfp4_codes"], ref["nvfp4_scales"])),
+                      (dq.FMT_LUT3, (ref["lut3_planes"], ref["lut3_scales"]))):
+        codes, scales, s = dq.export_canonical(w_imp, fmt)
+        assert np.array_equal(_np(codes).view(want[0].dtype), want[0]) and np.array_equal(_np(scales), want[1])
+        assert np.float32(_np(s)[0]) == np.float32(ref["s"])
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, 37).to(DEV)
+    sa = dq_inputs.static_act_scale(A.cpu())
+    assert torch.equal(dq.prefill_linear(w_imp, A, sa), dq.prefill_linear(w_pack, A, sa))
+    assert torch.equal(dq.decode_linear(w_imp, A[:3]), dq.decode_linear(w_pack, A[:3]))
+    # the LUT3-derived view from imported planes equals the oracle's autocast
+    w_view = dq.import_canonical(N, K, dq.FMT_NVFP4_FROM_LUT3, float(ref["s"]), lut3=lut)
+    codes, scales, _ = dq.export_canonical(w_view, dq.FMT_NVFP4_FROM_LUT3)
+    ac, asc = oracle.autocast_lut3_to_nvfp4(ref["lut3_planes"], ref["lut3_scales"])
+    assert np.array_equal(_np(codes), ac) and np.array_equal(_np(scales), asc)
+    with pytest.raises(dq.DQError):
+        dq.import_canonical(N, K, dq.FMT_NVFP4, float(ref["s"]), lut3=lut)      # missing NVFP4 buffers
+    _status_ok(dq)
+
+
 def test_custom_codebook(dq, oracle):
     N, K = 64, 256
     W, _ = _layer(oracle, N, K, 36)
