@@ -169,12 +169,129 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def run_stack(args):
+    """--workload c4_stack27b: the 64-layer 27B-class linear stack (fused qkv, o, fused gate/up, down per
+    layer; 23.15 G weights).  One step = one prefill pass of M = 4096 tokens through all 256 matrices
+    (activation quantiser + FP4 GEMM each; fresh N(0,1) input per matrix shape, no attention or
+    non-linearity in between) plus one decode token step over the same stack, replayed from one CUDA
+    graph as the paper measured decode (App. C.2).  Weights are drawn on the GPU (seeded) one matrix at a
+    time and packed immediately; the 23 GB packed stack is far larger than L2."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    import __graft_entry__ as g
+    if rank == 0:
+        g.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2609_26333_b200 as dq
+    from paper_2609_26333_b200 import replicas
+    peaks = load_peaks()
+    M, B = dq_inputs.C4_PREFILL_M, args.decode_batch
+    layers = args.layers or dq_inputs.C4_LAYERS
+    gen = torch.Generator(device=dev)
+    stack = []
+    t0 = time.perf_counter()
+    for layer in range(layers):
+        for cfg in dq_inputs.c4_fused_layer(layer):
+            gen.manual_seed(dq_inputs.seed_of(cfg, layer))
+            W = (torch.randn(cfg.N, cfg.K, generator=gen, device=dev, dtype=torch.float32) * cfg.w_std).to(torch.bfloat16)
+            stack.append((cfg, dq.pack_weights(W)))
+            del W
+    torch.cuda.synchronize()
+    pack_s = time.perf_counter() - t0
+    Ks = sorted({c.K for c, _ in stack})
+    Ns = sorted({c.N for c, _ in stack})
+    gen.manual_seed(4242)
+    A = {k: torch.randn(M, k, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16) for k in Ks}
+    X = {k: torch.randn(B, k, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16) for k in Ks}
+    sa = {k: dq_inputs.static_act_scale(A[k]) for k in Ks}
+    Y = {n: torch.empty(M, n, dtype=torch.bfloat16, device=dev) for n in Ns}
+    Yd = {n: torch.empty(B, n, dtype=torch.bfloat16, device=dev) for n in Ns}
+    ws_bytes = max(dq.prefill_workspace_bytes(w, M) for _, w in stack)
+    workspace = dq.alloc_workspace(ws_bytes, dev)
+
+    def prefill_pass():
+        for cfg, w in stack:
+            dq.prefill_quantize(w, A[cfg.K], sa[cfg.K], workspace)
+            dq.prefill_gemm(w, M, sa[cfg.K], Y[cfg.N], workspace)
+
+    def decode_pass():
+        for cfg, w in stack:
+            dq.decode_linear(w, X[cfg.K], out=Yd[cfg.N])
+
+    decode_pass()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        decode_pass()
+    for _ in range(max(3, args.warmup)):
+        prefill_pass()
+        graph.replay()
+    torch.cuda.synchronize()
+    steps = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    sampler = ClockSampler(local_rank)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    for i in range(steps):
+        ev[i][0].record()
+        prefill_pass()
+        ev[i][1].record()
+        graph.replay()
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    st, det = dq.get_status()
+    if st != 0:
+        raise RuntimeError(f"device status {dq.status_string(st)} (detail {det})")
+    p_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    d_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    p_ms, d_ms = replicas.max_over_ranks([p_ms, d_ms], device=dev)
+    weights = float(sum(c.N * c.K for c, _ in stack))
+    flops = 2.0 * M * weights
+    dec_bytes = 0.4375 * weights + sum(2.0 * B * (c.K + c.N) + 4 for c, _ in stack)
+    tflops = replicas.whole_job_rate(flops, world, p_ms) / 1e12
+    gbs = replicas.whole_job_rate(dec_bytes, world, d_ms) / 1e9
+    passes = (B + 1) // 2
+    line = {
+        "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": max(3, args.warmup),
+        "ms_per_step": p_ms + d_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "nvfp4",
+        "data": "synthetic",
+        "config": {"workload": "c4_stack27b", "layers": layers, "matrices": len(stack), "weights": weights, "M": M,
+                   "decode_batch": B, "parallelism": f"replicas x{world}",
+                   "l2": f"inputs larger than L2: packed stack {sum(w.packed.numel() for _, w in stack) / 1e9:.1f} GB",
+                   "step": "prefill pass (quantise + GEMM per matrix) + decode token step (one CUDA graph)"},
+        "clocks": clocks, "gpu_launches": steps * len(stack) * (2 + passes),
+        "prefill": {"ms": p_ms, "linear_tflops_per_gpu": tflops / world},
+        "decode": {"ms": d_ms, "value": gbs, "unit": "GB/s", "batch": B, "frac_of_measured_hbm": gbs / world / peaks["hbm_gbs"]},
+        "pack_s": pack_s,
+        "roofline": {"kernel": "gemm_nvfp4_pair_kernel (+ quant_act_kernel)", "bound": "tensor", "achieved": tflops / world,
+                     "peak": 4.0 * peaks["bf16_sustained"], "unit": "TFLOP/s",
+                     "frac": tflops / world / (4.0 * peaks["bf16_sustained"]), "traffic": None},
+    }
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(dq_inputs.CONFIGS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(dq_inputs.CONFIGS) + ["c4_stack27b"])
+    ap.add_argument("--layers", type=int, default=0, help="c4_stack27b only: number of layers (0 = all 64)")
     ap.add_argument("--mnk", default=None, help="M,N,K of an ad-hoc Gaussian layer (profiling small cases)")
     ap.add_argument("--impl", default="dq", choices=["dq", "reference"])
     ap.add_argument("--decode-batch", type=int, default=1)
@@ -185,6 +302,14 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "dq" else args.warmup
+    if args.workload == "c4_stack27b":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the stack workload is timed on the GPU arm only"}))
+            return
+        if args.steps == 200:
+            args.steps = 5
+        run_stack(args)
+        return
     cfg = dq_inputs.CONFIGS[args.workload]
     if args.mnk:
         m, n, k = (int(v) for v in args.mnk.split(","))
