@@ -36,6 +36,7 @@ namespace {
 
 constexpr int kRowsPerIter = 4;
 constexpr int kSmallCta = 512;                         // register budget of 128 per thread
+constexpr int kMidCta = 576;
 constexpr uint32_t kTableWindowAddr = 65536;          // table base inside the CTA's shared window (64 KiB aligned)
 constexpr uint32_t kTableBytes = 65536;               // 256 entries x 256 B
 constexpr uint32_t kDynSmemBytes = 231424;           // the whole opt-in shared memory of an SM less 1 KiB
@@ -401,6 +402,9 @@ cudaError_t launch_gemv_lut3(const GemvArgs &a, cudaStream_t stream)
         if (threads <= kSmallCta) {
             e = (B - b0 >= 2) ? launch_one<2, kSmallCta>(a, b0, grid, threads, W, G, S, stream)
                               : launch_one<1, kSmallCta>(a, b0, grid, threads, W, G, S, stream);
+        } else if (threads <= kMidCta) {               // 17 or 18 slices (K up to 18432): 112 registers per thread
+            e = (B - b0 >= 2) ? launch_one<2, kMidCta>(a, b0, grid, threads, W, G, S, stream)
+                              : launch_one<1, kMidCta>(a, b0, grid, threads, W, G, S, stream);
         } else {
             e = (B - b0 >= 2) ? launch_one<2, 1024>(a, b0, grid, threads, W, G, S, stream)
                               : launch_one<1, 1024>(a, b0, grid, threads, W, G, S, stream);
