@@ -183,6 +183,7 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
             cudaSuccess)
             return DQ_ERR_CUDA;
     }
+    if (dq::launch_pack_done(s) != cudaSuccess) return DQ_ERR_CUDA;
     dq_weights *w = new (std::nothrow) dq_weights;
     if (!w) return DQ_ERR_INTERNAL;
     w->magic = kMagic;
@@ -249,6 +250,7 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
             cudaSuccess)
             return DQ_ERR_CUDA;
     }
+    if (dq::launch_pack_done(s) != cudaSuccess) return DQ_ERR_CUDA;
     dq_weights *w = new (std::nothrow) dq_weights;
     if (!w) return DQ_ERR_INTERNAL;
     w->magic = kMagic;

@@ -127,6 +127,7 @@ cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, c
 cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                                int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
                                cudaStream_t stream);
+cudaError_t launch_pack_done(cudaStream_t stream);
 cudaError_t launch_set_scale(PackedHeader *hdr, float s, cudaStream_t stream);
 cudaError_t launch_import_nvfp4(const uint8_t *codes_in, const uint8_t *scales_in, int64_t N, int64_t K, uint8_t *codes,
                                 uint8_t *sf_swizzled, cudaStream_t stream);

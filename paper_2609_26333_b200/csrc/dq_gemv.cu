@@ -240,6 +240,13 @@ gemv_lut3_kernel(const uint8_t *__restrict__ lut, const uint8_t *__restrict__ ta
         }
     }
 
+    // Programmatic dependent launch: everything above touches only the packed weights, which no kernel
+    // running now can be writing (packing ends with a separate trailing launch).  Activations and output
+    // may belong to the kernel before this one in the stream, so wait for it here; the kernel after this
+    // one may begin its own set-up as soon as every CTA of this grid has got this far.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // this lane's 32 activations per batch column, widened to fp32 pairs, kept in registers
     unsigned long long xs[BT][16];
 #pragma unroll
@@ -369,10 +376,22 @@ static cudaError_t launch_one(const GemvArgs &a, int b0, int grid, int threads, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    gemv_lut3_kernel<BT, MAXT><<<grid, threads, kDynSmemBytes, stream>>>(
-        a.lut, a.table, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X), a.ldx, b0, (int)a.B,
-        reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy, (int)a.N, (int)a.K, W, G, S, a.status);
-    return cudaGetLastError();
+    // launched so that its set-up (barriers, lookup table, first weight blocks) may overlap the tail of
+    // the kernel before it in the stream; the kernel itself waits before it touches X or Y
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = kDynSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_lut3_kernel<BT, MAXT>, a.lut, a.table, a.hdr,
+                              reinterpret_cast<const __nv_bfloat16 *>(a.X), (int64_t)a.ldx, b0, (int)a.B,
+                              reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N, (int)a.K, W, G, S,
+                              a.status);
 }
 
 cudaError_t launch_gemv_lut3(const GemvArgs &a, cudaStream_t stream)

@@ -374,6 +374,16 @@ cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, 
     return cudaGetLastError();
 }
 
+// Last launch of every pack / import: does nothing.  The decode kernel is launched so that its set-up may
+// overlap the kernel before it in the stream; with this launch in between, that kernel is never one that
+// writes the packed buffer.
+__global__ void pack_done_kernel() {}
+cudaError_t launch_pack_done(cudaStream_t stream)
+{
+    pack_done_kernel<<<1, 32, 0, stream>>>();
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ import
 
 // Canonical codes / scales (the layouts of the export) -> device layouts.  Inverse of the export kernels.
