@@ -203,6 +203,11 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     cluster_sync_all();            // both CTAs' barriers exist before anyone signals across the pair
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    // Programmatic dependent launch: the set-up above may overlap the tail of the kernel before this one
+    // (normally the activation quantiser, whose output this kernel reads); nothing is loaded or stored
+    // before that kernel has completed.  A dependent kernel may start its own set-up from here on.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int tiles_m = (M + 2 * BM - 1) / (2 * BM);
     const int tiles_n = (N + BN - 1) / BN;
@@ -467,10 +472,19 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
     int pairs = sms / 2;
     if (tiles < pairs) pairs = tiles;
-    gemm_nvfp4_pair_kernel<<<2 * pairs, kThreads, SMEM_BYTES, stream>>>(
-        tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr, a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy,
-        (int)a.M, (int)a.N, (int)a.K, a.status, a.probe);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3((unsigned)kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+                              a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M, (int)a.N,
+                              (int)a.K, a.status, a.probe);
 }
 
 }  // namespace dq

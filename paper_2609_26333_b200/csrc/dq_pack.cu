@@ -503,6 +503,10 @@ template <bool SWIZZLED>
 __global__ void __launch_bounds__(256) quant_act_kernel(const __nv_bfloat16 *A, int64_t M, int64_t K, int64_t lda,
                                                         float s, uint8_t *codes, uint8_t *sf)
 {
+    // launched with programmatic stream serialization (hides the launch latency behind the previous
+    // kernel); that kernel may produce A or still read the workspace, so wait for it before anything else
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t nb = K / 16;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool live = i < M * nb;
@@ -533,9 +537,17 @@ cudaError_t launch_quant_act(const void *A_bf16, int64_t M, int64_t K, int64_t l
     const int64_t total = M * (K / 16);
     const unsigned blocks = (unsigned)((total + 255) / 256);
     const __nv_bfloat16 *A = reinterpret_cast<const __nv_bfloat16 *>(A_bf16);
-    if (swizzled) quant_act_kernel<true><<<blocks, 256, 0, stream>>>(A, M, K, lda, act_scale, codes, sf);
-    else quant_act_kernel<false><<<blocks, 256, 0, stream>>>(A, M, K, lda, act_scale, codes, sf);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (swizzled) return cudaLaunchKernelEx(&cfg, quant_act_kernel<true>, A, M, K, lda, act_scale, codes, sf);
+    return cudaLaunchKernelEx(&cfg, quant_act_kernel<false>, A, M, K, lda, act_scale, codes, sf);
 }
 
 }  // namespace dq
