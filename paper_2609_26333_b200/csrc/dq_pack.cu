@@ -500,54 +500,60 @@ __device__ __forceinline__ uint32_t quant_block_nvfp4_bf16(const uint32_t (&w)[8
 // 16-block: 32 B in, 8 B of codes out; four neighbouring lanes (one 64-wide k
 // atom) merge their scale bytes into one 32-bit store of the MMA scale layout.
 template <bool SWIZZLED>
-__global__ void __launch_bounds__(256) quant_act_kernel(const __nv_bfloat16 *A, int64_t M, int64_t K, int64_t lda,
+__global__ void __launch_bounds__(256) quant_act_kernel(const __nv_bfloat16 *A, int M, int nb, int64_t lda,
                                                         float s, uint8_t *codes, uint8_t *sf)
 {
     // launched with programmatic stream serialization (hides the launch latency behind the previous
     // kernel); that kernel may produce A or still read the workspace, so wait for it before anything else
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int64_t nb = K / 16;
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool live = i < M * nb;
-    const int64_t r = live ? i / nb : 0, b = live ? i % nb : 0;
+    // 64 blocks of one row per 64 threads, four rows per CTA: no division, 32-bit index arithmetic
+    const int b = blockIdx.y * 64 + threadIdx.x;
+    const int r = blockIdx.x * 4 + threadIdx.y;
+    const bool live = (b < nb) && (r < M);
     const float rc6 = __frcp_rn(__fmul_rn(6.0f, s));
     uint32_t d8 = 0;
     if (live) {
-        const uint4 *p = reinterpret_cast<const uint4 *>(A + r * lda + b * 16);
+        const uint4 *p = reinterpret_cast<const uint4 *>(A + (int64_t)r * lda + b * 16);
         const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
         const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         uint2 c;
         d8 = quant_block_nvfp4_bf16(w, s, rc6, c);
-        *reinterpret_cast<uint2 *>(codes + r * (K / 2) + b * 8) = c;
+        *reinterpret_cast<uint2 *>(codes + ((int64_t)r * nb + b) * 8) = c;
     }
     // K % 64 == 0, so lanes 4q..4q+3 always hold the four blocks of one k atom of one row
     uint32_t w = d8 << (8 * (threadIdx.x & 3));
     w |= __shfl_xor_sync(0xffffffffu, w, 1);
     w |= __shfl_xor_sync(0xffffffffu, w, 2);
     if (live && (threadIdx.x & 3) == 0) {
-        if (SWIZZLED) *reinterpret_cast<uint32_t *>(sf + sf_swizzled_offset(r, b, K)) = w;
-        else *reinterpret_cast<uint32_t *>(sf + r * nb + b) = w;
+        if (SWIZZLED) {
+            // atom (r / 128, b / 4) of 512 bytes; row rr of the atom at (rr % 32) * 16 + (rr / 32) * 4
+            const int rr = r & 127;
+            const size_t off = ((size_t)(r >> 7) * (size_t)(nb >> 2) + (size_t)(b >> 2)) * 512 + (size_t)((rr & 31) * 16 + (rr >> 5) * 4);
+            *reinterpret_cast<uint32_t *>(sf + off) = w;
+        } else {
+            *reinterpret_cast<uint32_t *>(sf + (int64_t)r * nb + b) = w;
+        }
     }
 }
 
 cudaError_t launch_quant_act(const void *A_bf16, int64_t M, int64_t K, int64_t lda, float act_scale, uint8_t *codes,
                              uint8_t *sf, int swizzled, cudaStream_t stream)
 {
-    const int64_t total = M * (K / 16);
-    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const int nb = (int)(K / 16);
+    const int m = (int)M;
     const __nv_bfloat16 *A = reinterpret_cast<const __nv_bfloat16 *>(A_bf16);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(blocks);
-    cfg.blockDim = dim3(256);
+    cfg.gridDim = dim3((unsigned)((m + 3) / 4), (unsigned)((nb + 63) / 64));
+    cfg.blockDim = dim3(64, 4);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (swizzled) return cudaLaunchKernelEx(&cfg, quant_act_kernel<true>, A, M, K, lda, act_scale, codes, sf);
-    return cudaLaunchKernelEx(&cfg, quant_act_kernel<false>, A, M, K, lda, act_scale, codes, sf);
+    if (swizzled) return cudaLaunchKernelEx(&cfg, quant_act_kernel<true>, A, m, nb, lda, act_scale, codes, sf);
+    return cudaLaunchKernelEx(&cfg, quant_act_kernel<false>, A, m, nb, lda, act_scale, codes, sf);
 }
 
 }  // namespace dq
