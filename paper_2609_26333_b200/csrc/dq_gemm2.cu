@@ -149,9 +149,8 @@ __device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volati
 
 // pair-tile index -> (256-row block, 256-column block); m fastest inside groups of 8 so that the
 // pairs running together share W column blocks and A row blocks in L2
-__device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, int &mb, int &nb)
+__device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, int &mb, int &nb, int GM)
 {
-    constexpr int GM = 8;
     const int per_group = GM * tiles_n;
     const int g = t / per_group;
     const int first_m = g * GM;
@@ -165,7 +164,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
                        const __grid_constant__ CUtensorMap tmap_y, const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
-                       int64_t ldy, int M, int N, int K, StatusWord *status, int probe)
+                       int64_t ldy, int M, int N, int K, StatusWord *status, int probe, int group_m)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -216,6 +215,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const int num_ks = (katoms + kKbPerStage - 1) / kKbPerStage;
     const int pair = blockIdx.x >> 1;
     const int npairs = gridDim.x >> 1;
+    const int gm = (probe >> 8) > 0 ? (probe >> 8) : group_m;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -224,7 +224,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             bool ok = true;
             for (int t = pair; t < num_tiles && ok; t += npairs) {
                 int mb, nb;
-                tile_coords2(t, tiles_m, tiles_n, mb, nb);
+                tile_coords2(t, tiles_m, tiles_n, mb, nb, gm);
                 const int rowblk = mb * 2 + (int)rank;            // 128-row block of A this CTA owns
                 for (int ks = 0; ks < num_ks; ++ks) {
                     if (!mbar_wait2(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
@@ -342,7 +342,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         bool ok = true;
         for (int t = pair; t < num_tiles && ok; t += npairs) {
             int mb, nb;
-            tile_coords2(t, tiles_m, tiles_n, mb, nb);
+            tile_coords2(t, tiles_m, tiles_n, mb, nb, gm);
             if (!mbar_wait2(tmem_full_bar, acc_phase, abort_flag, peer_abort)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(half * 128);
@@ -472,6 +472,10 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
     int pairs = sms / 2;
     if (tiles < pairs) pairs = tiles;
+    // Tile order: groups of group_m row tiles sweep all column tiles, so that the A rows of a group stay in L2
+    // while each W tile is read once per group.  Largest power of two whose A codes + scales fit about 48 MB.
+    int group_m = 4;
+    while (group_m < 64 && (double)(2 * group_m) * 256.0 * (double)a.K * 0.5625 <= 48.0e6) group_m *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3((unsigned)kThreads);
@@ -484,7 +488,7 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                               a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M, (int)a.N,
-                              (int)a.K, a.status, a.probe);
+                              (int)a.K, a.status, a.probe, group_m);
 }
 
 }  // namespace dq
