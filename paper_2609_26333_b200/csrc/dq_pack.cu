@@ -281,41 +281,56 @@ cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, i
 
 // NVFP4 view of the LUT3 codes (Sec. 2.3): level -> nearest E2M1 value, element signs
 // flipped under a negative block scale, block scale |d|, same tensor scale.
-__global__ void autocast_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
-                                int64_t K, uint8_t *codes, uint8_t *sf)
+// One thread per plane word (32 weights).  The three plane words are merged into bytes that hold the six
+// index bits of a weight pair (as in the decode kernel); a 64-entry shared-memory table maps such a byte to
+// the byte of two E2M1 codes, in three variants: positive scale, negative scale (sign bits of non-zero codes
+// flipped), zero scale (all codes zero).  Pair q = 4g + j of the word is byte j of the word rotated by 2g,
+// and is output byte q of the row's 16 code bytes, so each merged word gives one output word.
+__global__ void __launch_bounds__(256) autocast_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
+                                                       int64_t K, uint8_t *codes, uint8_t *sf)
 {
-    const int64_t nw = K / 32;
+    __shared__ uint8_t table[3][64];                // [variant][pair pattern] -> two E2M1 codes
+    const uint32_t amap = hdr->autocast_map;
+    if (threadIdx.x < 192) {
+        const int v = threadIdx.x >> 6, e = threadIdx.x & 63;
+        const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
+        const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
+        uint32_t ca = (amap >> (4 * ia)) & 0xFu, cb = (amap >> (4 * ib)) & 0xFu;
+        if (v == 1) { if (ca & 7u) ca ^= 8u; if (cb & 7u) cb ^= 8u; }
+        if (v == 2) { ca = 0u; cb = 0u; }
+        table[v][e] = (uint8_t)(ca | (cb << 4));
+    }
+    __syncthreads();
+    const int nw = (int)(K / 32);
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N * nw) return;
-    const int64_t r = i / nw, j = i % nw;
-    const uint32_t amap = hdr->autocast_map;
+    const int64_t r = i / nw;
+    const int j = (int)(i - r * nw);
     const uint32_t p0 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 0, K));
     const uint32_t p1 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 1, K));
     const uint32_t p2 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 2, K));
-    uint32_t out[4] = {0, 0, 0, 0};
+    const uint32_t d2 = *reinterpret_cast<const unsigned short *>(lut + lut_scale_offset(r, j * 2, K));
+    uint32_t out[4];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const uint32_t d8 = lut[lut_scale_offset(r, j * 2 + h, K)];
-        sf[sf_swizzled_offset(r, j * 2 + h, K)] = (uint8_t)(d8 & 0x7Fu);
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const int bit = h * 16 + q;
-            const uint32_t idx = ((p0 >> lut3_bitpos(0, bit)) & 1u) | (((p1 >> lut3_bitpos(1, bit)) & 1u) << 1) |
-                                 (((p2 >> lut3_bitpos(2, bit)) & 1u) << 2);
-            uint32_t c = (amap >> (4 * idx)) & 0xFu;
-            if ((d8 & 0x80u) && (c & 0x7u)) c ^= 0x8u;
-            if (d8 == 0u) c = 0u;
-            out[bit / 8] |= c << (4 * (bit % 8));
-        }
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t d8 = (g < 2) ? (d2 & 0xFFu) : (d2 >> 8);            // pairs 0..7 are block 0, 8..15 block 1
+        const uint8_t *tab = table[d8 == 0u ? 2 : ((d8 & 0x80u) ? 1 : 0)];
+        const uint32_t a = __funnelshift_r(p0, p0, 2 * g), b = __funnelshift_r(p1, p1, 2 * g),
+                       c = __funnelshift_r(p2, p2, 2 * g);
+        const uint32_t u = (a & 0x03030303u) | (b & 0x0C0C0C0Cu) | (c & 0x30303030u);
+        out[g] = (uint32_t)tab[u & 0xFFu] | ((uint32_t)tab[(u >> 8) & 0xFFu] << 8) |
+                 ((uint32_t)tab[(u >> 16) & 0xFFu] << 16) | ((uint32_t)tab[u >> 24] << 24);
     }
-    *reinterpret_cast<uint4 *>(codes + r * (K / 2) + j * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+    *reinterpret_cast<uint4 *>(codes + r * (K / 2) + (int64_t)j * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+    sf[sf_swizzled_offset(r, j * 2, K)] = (uint8_t)(d2 & 0x7Fu);
+    sf[sf_swizzled_offset(r, j * 2 + 1, K)] = (uint8_t)((d2 >> 8) & 0x7Fu);
 }
 
 cudaError_t launch_autocast(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                             int64_t K, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream)
 {
     const int64_t total = N * (K / 32);
-    autocast_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(hdr, lut_dev, N, K, codes, sf_swizzled);
+    autocast_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, lut_dev, N, K, codes, sf_swizzled);
     return cudaGetLastError();
 }
 
