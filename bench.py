@@ -411,6 +411,31 @@ def main():
     if st != 0:
         raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the timed region")
 
+    # ---- decode launches back to back (token after token, rotating weight copies): the events of the
+    #      step loop separate the launches, which hides the overlap of one launch's set-up with the tail
+    #      of the launch before it (programmatic dependent launch); this loop shows it
+    nb2b = max(50, 3 * copies)
+    for i in range(copies):
+        dq.decode_linear(ws[i], X, out=Yd)
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    b0.record()
+    for i in range(nb2b):
+        dq.decode_linear(ws[i % copies], X, out=Yd)
+    b1.record()
+    torch.cuda.synchronize()
+    d_b2b_ms = b0.elapsed_time(b1) / nb2b
+    # the same token loop on the NVFP4 view (weight-only NVFP4A16 decode, 0.5625 byte per weight)
+    for i in range(copies):
+        dq.decode_linear_nvfp4(ws[i], X, out=Yd)
+    torch.cuda.synchronize()
+    b0.record()
+    for i in range(nb2b):
+        dq.decode_linear_nvfp4(ws[i % copies], X, out=Yd)
+    b1.record()
+    torch.cuda.synchronize()
+    d_nv_ms = b0.elapsed_time(b1) / nb2b
+
     # ---- end to end: pinned host buffers, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -447,8 +472,9 @@ def main():
 
     # ---- max over ranks ----
     from paper_2609_26333_b200 import replicas
-    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms = replicas.max_over_ranks(
-        [total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0, e2e["decode_ms"] if e2e else 0.0], device=dev)
+    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms, d_b2b_ms = replicas.max_over_ranks(
+        [total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0, e2e["decode_ms"] if e2e else 0.0, d_b2b_ms],
+        device=dev)
 
     flops = 2.0 * M * N * K
     dec_bytes = 0.4375 * N * K + 2.0 * B * K + 2.0 * B * N + 4
@@ -473,7 +499,12 @@ def main():
                     "linear_tflops_per_gpu": prefill_tflops / world, "quant_gbs": quant_gbs,
                     "quant_frac_of_hbm": quant_gbs / peaks["hbm_gbs"]},
         "decode": {"ms": d_ms, "value": world * decode_gbs, "unit": "GB/s", "batch": B,
-                   "frac_of_measured_hbm": decode_gbs / peaks["hbm_gbs"], "frac_of_8tbs": decode_gbs / 8000.0},
+                   "frac_of_measured_hbm": decode_gbs / peaks["hbm_gbs"], "frac_of_8tbs": decode_gbs / 8000.0,
+                   "back_to_back_ms": d_b2b_ms, "back_to_back_gbs": world * dec_bytes / (d_b2b_ms * 1e-3) / 1e9,
+                   "back_to_back_frac_of_measured_hbm": dec_bytes / (d_b2b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "decode_nvfp4a16": {"back_to_back_ms": d_nv_ms, "unit": "GB/s",
+                            "value": world * (0.5625 * N * K + 2.0 * B * (K + N)) / (d_nv_ms * 1e-3) / 1e9,
+                            "frac_of_measured_hbm": (0.5625 * N * K + 2.0 * B * (K + N)) / (d_nv_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "pack_ms": pack_ms,
         "roofline": {"kernel": "gemm_nvfp4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,

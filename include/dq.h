@@ -167,6 +167,17 @@ int dq_prefill_linear_static(const dq_weights *w, const void *A_dev, int64_t M, 
 int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
                      void *Y_dev, int64_t ldy, void *stream);
 
+/*
+ * The same decode on the handle's NVFP4 view (weight-only NVFP4A16, Sec. 2.3 and Table 1
+ * "format-disaggregated NVFP4": one stored 4.5-bit matrix serves the tensor-core prefill and
+ * this mat-vec):
+ *   Y[b][n] = bf16( sum_k X[b][k] * W^[n][k] ),  W^ = s * d_b * e2m1(code),
+ * raw bf16 activations, fp32 accumulation.  Needs DQ_FMT_NVFP4 or DQ_FMT_NVFP4_FROM_LUT3 in the
+ * handle (DQ_ERR_INVALID_ARG otherwise).  Arguments and limits as dq_decode_linear.
+ */
+int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
+                           void *Y_dev, int64_t ldy, void *stream);
+
 /* ---- parity hooks: canonical encodings, compared bit for bit with the oracle ---- */
 
 /*

@@ -285,6 +285,14 @@ def prefill_linear(A_f32, act_scale: float, nv_codes, nv_scales, s_w: float, row
     return matmul_nt_lib(Ah, Wh) if lib_matmul else matmul_nt(Ah, Wh)
 
 
+def decode_linear_nvfp4(X_f32, nv_codes, nv_scales, s_w: float, lib_matmul=True):
+    """Decode on the NVFP4 view (weight-only NVFP4A16, Sec. 2.3 / Table 1): raw bf16 activations
+    times NVFP4-dequantised weights, fp64."""
+    X = np.asarray(X_f32, dtype=np.float64)
+    Wh = dequant_nvfp4(nv_codes, nv_scales, s_w)
+    return matmul_nt_lib(X, Wh) if lib_matmul else matmul_nt(X, Wh)
+
+
 def decode_linear(X_f32, planes, lut_scales, s_w: float, codebook_f16=None, lib_matmul=True):
     """Decode: raw bf16 activations times LUT3-dequantised weights, fp64 (App. C.2)."""
     X = np.asarray(X_f32, dtype=np.float64)

@@ -20,7 +20,7 @@ DT_FP32 = 1
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
-           "dq_decode_linear", "dq_export_canonical", "dq_import_canonical",
+           "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
 
 
@@ -65,6 +65,8 @@ def lib() -> C.CDLL:
         L.dq_prefill_linear_static.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp]
         L.dq_decode_linear.restype = C.c_int
         L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_decode_linear_nvfp4.restype = C.c_int
+        L.dq_decode_linear_nvfp4.argtypes = [vp, vp, i64, i64, vp, i64, vp]
         L.dq_import_canonical.restype = C.c_int
         L.dq_import_canonical.argtypes = [C.c_int64, C.c_int64, C.c_uint, vp, vp, vp, vp, C.c_float,
                                           C.POINTER(C.c_uint16), vp, C.c_size_t, vp, C.POINTER(vp)]
@@ -240,6 +242,17 @@ def decode_linear(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None, strea
         out = torch.empty(B, w.N, dtype=torch.bfloat16, device=X.device)
     _check(lib().dq_decode_linear(w.handle, X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
                                   _stream_ptr(stream)), "dq_decode_linear")
+    return out
+
+
+def decode_linear_nvfp4(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """dq_decode_linear_nvfp4: Y = X @ NVFP4(W)^T (weight-only NVFP4A16), bf16 out, batch 1..64."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    B = X.shape[0]
+    if out is None:
+        out = torch.empty(B, w.N, dtype=torch.bfloat16, device=X.device)
+    _check(lib().dq_decode_linear_nvfp4(w.handle, X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
+                                        _stream_ptr(stream)), "dq_decode_linear_nvfp4")
     return out
 
 

@@ -183,6 +183,8 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
             cudaSuccess)
             return DQ_ERR_CUDA;
     }
+    if ((formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3)) && dq::launch_fill_e2m1_table(s) != cudaSuccess)
+        return DQ_ERR_CUDA;
     if (dq::launch_pack_done(s) != cudaSuccess) return DQ_ERR_CUDA;
     dq_weights *w = new (std::nothrow) dq_weights;
     if (!w) return DQ_ERR_INTERNAL;
@@ -250,6 +252,8 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
             cudaSuccess)
             return DQ_ERR_CUDA;
     }
+    if ((formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3)) && dq::launch_fill_e2m1_table(s) != cudaSuccess)
+        return DQ_ERR_CUDA;
     if (dq::launch_pack_done(s) != cudaSuccess) return DQ_ERR_CUDA;
     dq_weights *w = new (std::nothrow) dq_weights;
     if (!w) return DQ_ERR_INTERNAL;
@@ -373,6 +377,33 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
     st = dq_prefill_quantize(w, A_dev, M, lda, act_global_scale, workspace_dev, workspace_bytes, stream);
     if (st != DQ_OK) return st;
     return dq_prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream);
+}
+
+int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                           void *stream)
+{
+    if (!valid_handle(w) || !X_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
+    if (!has_nvfp4_view(w)) return DQ_ERR_INVALID_ARG;
+    if (B < 1 || B > 64) return DQ_ERR_INVALID_ARG;
+    if (ldx < w->K || ldy < w->N || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
+    if (!aligned(X_dev, 16) || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    dq::GemvNvArgs g;
+    g.codes = w->base + w->layout.nv_codes_off;
+    g.sf = w->base + w->layout.nv_sf_off;
+    g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
+    g.status = status_word_ptr();
+    if (!g.status) return DQ_ERR_CUDA;
+    g.X = X_dev;
+    g.ldx = ldx;
+    g.B = B;
+    g.Y = Y_dev;
+    g.ldy = ldy;
+    g.N = w->N;
+    g.K = w->K;
+    if (dq::launch_gemv_nvfp4(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
 }
 
 int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,

@@ -162,4 +162,15 @@ struct GemvArgs {
 };
 cudaError_t launch_gemv_lut3(const GemvArgs &args, cudaStream_t stream);
 
+struct GemvNvArgs {
+    const uint8_t *codes; const uint8_t *sf;              // NVFP4 view: [N][K/2] codes, MMA-layout scales
+    const PackedHeader *hdr;
+    StatusWord *status = nullptr;
+    const void *X; int64_t ldx; int64_t B;
+    void *Y; int64_t ldy;
+    int64_t N, K;
+};
+cudaError_t launch_gemv_nvfp4(const GemvNvArgs &args, cudaStream_t stream);
+cudaError_t launch_fill_e2m1_table(cudaStream_t stream);   // value-pair table of the NVFP4 decode kernel
+
 }  // namespace dq

@@ -283,6 +283,27 @@ def test_decode_parity(dq, oracle, N, K, seed, B):
     check_outputs(_f64(Y), Yr, S, f"decode {B}x{N}x{K}")
 
 
+@pytest.mark.parametrize("N,K,seed", [(512, 256, 0), (144, 384, 31), (784, 1152, 32), (272, 17408, 33)])
+@pytest.mark.parametrize("B", [1, 2, 3, 8])
+def test_decode_nvfp4_parity(dq, oracle, N, K, seed, B):
+    """Weight-only decode on the NVFP4 view; also from the LUT3-derived view of the same matrix."""
+    W, ref = _layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    X = dq_inputs.gaussian_bf16(B, K, 1.0, 1000 + seed + B)
+    Y = dq.decode_linear_nvfp4(w, X.to(DEV))
+    _status_ok(dq)
+    Yr, S = oracle.decode_linear_nvfp4(dq_inputs.bf16_to_f32_numpy(X), ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, f"nvfp4 decode {B}x{N}x{K}")
+    if B == 2 and K <= 1152:
+        w2 = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4_FROM_LUT3)
+        ac, asc = oracle.autocast_lut3_to_nvfp4(ref["lut3_planes"], ref["lut3_scales"])
+        Yr, S = oracle.decode_linear_nvfp4(dq_inputs.bf16_to_f32_numpy(X), ac, asc, ref["s"])
+        check_outputs(_f64(dq.decode_linear_nvfp4(w2, X.to(DEV))), Yr, S, "nvfp4 decode on the LUT3-derived view")
+        w3 = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+        with pytest.raises(dq.DQError):
+            dq.decode_linear_nvfp4(w3, X.to(DEV))
+
+
 def test_decode_one_hot_and_strided(dq, oracle):
     N, K = 256, 512
     W, ref = _layer(oracle, N, K, 64)

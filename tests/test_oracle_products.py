@@ -87,3 +87,29 @@ def test_tiny_config_against_independent_loop_and_library_matmul(oracle):
     Yfull = W.astype(np.float64) @ x[0].astype(np.float64)
     rel = np.linalg.norm(Yd[0] - Yfull) / np.linalg.norm(Yfull)
     assert 0.05 < rel < 0.3
+
+
+def test_nvfp4_decode_is_activations_times_dequantised_weights(oracle):
+    """Weight-only decode on the NVFP4 view (Sec. 2.3): a one-hot activation picks one dequantised
+    column, an all-ones activation gives row sums of s * d * e2m1 evaluated here from the printed value set,
+    and the triple-loop and library products agree."""
+    rng = np.random.default_rng(11)
+    N, K = 48, 128
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    ref = oracle.pack_weights(W)
+    codes, scales, s = ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"]
+    e2m1 = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)          # App. A.3 "NVFP4"
+    lo, hi = codes & 0xF, codes >> 4
+    nib = np.stack([lo, hi], axis=-1).reshape(N, K)
+    vals = np.where(nib & 8, -1.0, 1.0) * e2m1[nib & 7]
+    sc = scales.astype(np.uint32)
+    e, m = (sc >> 3) & 15, sc & 7
+    d = np.where(e > 0, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7), m / 8.0 * 2.0 ** -6)
+    What = np.float64(np.float32(s)) * np.repeat(d, 16, axis=1) * vals
+    X = np.zeros((3, K)); X[0, 5] = 1.0; X[1, 127] = -2.0; X[2, :] = 1.0
+    Y, S = oracle.decode_linear_nvfp4(X, codes, scales, s, lib_matmul=False)
+    assert np.array_equal(Y[0], What[:, 5]) and np.array_equal(Y[1], -2.0 * What[:, 127])
+    assert np.allclose(Y[2], What.sum(axis=1), rtol=1e-13, atol=1e-15)
+    assert np.allclose(S[2], np.abs(What).sum(axis=1), rtol=1e-13)
+    Y2, _ = oracle.decode_linear_nvfp4(X, codes, scales, s, lib_matmul=True)
+    assert np.allclose(Y, Y2, rtol=1e-13, atol=1e-15)
