@@ -24,6 +24,7 @@ namespace dq {
 namespace {
 
 constexpr int kRows = 4;                                  // rows per work unit
+constexpr int kSlots = 4;                                 // cross-warp reduction slots per row group
 constexpr uint32_t kTableWindowAddr = 65536;              // table base in the CTA's shared window (64 KiB aligned)
 constexpr uint32_t kTableBytes = 65536;                   // 256 entries x 32 lane slots x (fp32, fp32)
 constexpr uint32_t kDynSmemBytes = 2 * 65536;             // [control + reduction | table]
@@ -84,9 +85,10 @@ gemv_nvfp4_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restrict__
 {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
-    float *red = reinterpret_cast<float *>(smem_raw);                         // [G][2][rows][BT][W] partial sums
+    float *red = reinterpret_cast<float *>(smem_raw);                         // [G][kSlots][rows][BT][W] partial sums
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + 32768);
     const uint32_t table_bar = win0 + 32768 + 64;
+    volatile int *sync_words = reinterpret_cast<volatile int *>(smem_raw + 32768 + 128);   // [G][kSlots] x (generation, count)
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -96,12 +98,12 @@ gemv_nvfp4_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restrict__
     const int widx = w * 32 + lane;
     const bool active = widx < pieces;
     const int katoms = K / 64;
-    const int group_threads = W * 32;
 
-    if (win0 + 32768 + 128 > kTableWindowAddr || (size_t)G * 2 * kRows * BT * W * sizeof(float) > 32768) {
+    if (win0 + 32768 + 128 + 16 * kSlots * 8 > kTableWindowAddr || (size_t)G * kSlots * kRows * BT * W * sizeof(float) > 32768) {
         if (threadIdx.x == 0) { atomicExch(&status->status, (int)DQ_ERR_INTERNAL); atomicExch(&status->detail, 0x32000); }
         return;
     }
+    if (threadIdx.x < 16 * kSlots * 2) sync_words[threadIdx.x] = 0;
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         tc::mbar_init(table_bar, 1);
@@ -221,19 +223,48 @@ gemv_nvfp4_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restrict__
             v[0][t] += __shfl_xor_sync(0xffffffffu, v[0][t], 2);
             v[0][t] += __shfl_xor_sync(0xffffffffu, v[0][t], 1);
         }
-        float *rbuf = red + ((grp * 2 + (it & 1)) * kRows * BT) * W;
+        // Cross-warp sum without a barrier: every warp of the group drops its partial sums into slot it % kSlots
+        // and bumps the slot's counter; the warp that arrives last adds the W partials in a fixed order (so the
+        // result does not depend on arrival order), stores the outputs and frees the slot for iteration it + kSlots.
+        const int slot = it & (kSlots - 1);
+        volatile int *gen = sync_words + (grp * kSlots + slot) * 2;
+        int *cnt = const_cast<int *>(gen) + 1;
+        if (ok) {
+            uint32_t good = 1;
+            if (lane == 0) {
+                const int want = it / kSlots;
+                long long t0 = 0;
+                uint32_t spins = 0;
+                while (*gen != want) {
+                    if ((++spins & 255u) == 0u) {
+                        if (t0 == 0) t0 = clock64();
+                        if (*abort_flag || clock64() - t0 > tc::kWaitBudgetCycles) { *abort_flag = 1; good = 0; break; }
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+        }
+        float *rbuf = red + ((grp * kSlots + slot) * kRows * BT) * W;
         if ((lane & 7) == 0) {
             const int row_l = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
 #pragma unroll
             for (int t = 0; t < BT; ++t) rbuf[(row_l * BT + t) * W + w] = v[0][t];
         }
-        asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(group_threads) : "memory");
-        if (w == 0 && lane < kRows * BT) {
-            const int row_l = lane / BT, t = lane % BT;
-            float tot = 0.0f;
-            for (int ww = 0; ww < W; ++ww) tot += rbuf[(row_l * BT + t) * W + ww];
-            const int row = (u >> 5) * 128 + (u & 31) + 32 * row_l;
-            if (b0 + t < B && row < N) Y[(int64_t)(b0 + t) * ldy + row] = __float2bfloat16_rn(tot * s_w);
+        __syncwarp();
+        int prev = 0;
+        if (lane == 0) { __threadfence_block(); prev = atomicAdd(cnt, 1); }
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev == W - 1) {
+            __threadfence_block();
+            if (lane < kRows * BT) {
+                const int row_l = lane / BT, t = lane % BT;
+                float tot = 0.0f;
+                for (int ww = 0; ww < W; ++ww) tot += reinterpret_cast<volatile float *>(rbuf)[(row_l * BT + t) * W + ww];
+                const int row = (u >> 5) * 128 + (u & 31) + 32 * row_l;
+                if (ok && b0 + t < B && row < N) Y[(int64_t)(b0 + t) * ldy + row] = __float2bfloat16_rn(tot * s_w);
+            }
+            __syncwarp();
+            if (lane == 0) { *cnt = 0; __threadfence_block(); *gen = it / kSlots + 1; }
         }
         cur = nxt;
     }
