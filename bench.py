@@ -441,20 +441,17 @@ def main():
     if not args.no_e2e:
         Y_host = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
         Yd_host = torch.empty(B, N, dtype=torch.bfloat16).pin_memory()
-        A2, X2 = torch.empty_like(A), torch.empty_like(X)
+        staging = dq.alloc_workspace(dq.prefill_host_staging_bytes(ws[0], M), dev)
 
         def e2e_step(i, ev=None):
+            # the C-ABI calls on host buffers: copies in both directions are inside the calls
             w = ws[i % copies]
             if ev is not None:
                 ev[0].record()
-            A2.copy_(A_host, non_blocking=True)
-            dq.prefill_linear(w, A2, sa, out=Y, workspace=workspace)
-            Y_host.copy_(Y, non_blocking=True)
+            dq.prefill_linear_host(w, A_host, sa, Y_host, staging)
             if ev is not None:
                 ev[1].record()
-            X2.copy_(X_host, non_blocking=True)
-            dq.decode_linear(w, X2, out=Yd)
-            Yd_host.copy_(Yd, non_blocking=True)
+            dq.decode_linear_host(w, X_host, Yd_host, staging)
             if ev is not None:
                 ev[2].record()
 

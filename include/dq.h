@@ -178,6 +178,33 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
 int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
                            void *Y_dev, int64_t ldy, void *stream);
 
+/* ---- host-buffer entry points (the paper has no counterpart; they exist to use and to measure the path
+ *      end to end through this interface, copies included) ---- */
+
+/*
+ * dq_prefill_linear on host memory: A_host (M x K bf16, row stride lda) is copied to the device, the
+ * prefill linear runs, Y_host (M x N bf16, row stride ldy) receives the result.  M is cut into row
+ * chunks; the copy in of the next chunk and the copy out of the previous one overlap the kernels of the
+ * current one on two internal streams per device (created at the first call on that device, which
+ * therefore must not happen during a stream capture; these calls are not capturable at all).
+ * A_host and Y_host should be pinned (cudaHostAlloc / cudaHostRegister), else the copies serialise.
+ * staging_dev: caller-owned device buffer of at least dq_prefill_host_staging_bytes(w, M) bytes
+ * (device copies of A and Y plus the prefill workspace of one chunk), 1024-byte aligned.
+ * On return everything is queued; `stream` is complete when Y_host is.  All calls on one device share
+ * the internal streams and events: issue them from one thread, ordered on the caller's streams.
+ */
+int dq_prefill_host_staging_bytes(const dq_weights *w, int64_t M, size_t *bytes_host);
+int dq_prefill_linear_host(const dq_weights *w, const void *A_host, int64_t M, int64_t lda,
+                           float act_global_scale, void *Y_host, int64_t ldy, void *staging_dev,
+                           size_t staging_bytes, void *stream);
+
+/*
+ * dq_decode_linear on host memory (X_host B x K, Y_host B x N, bf16): copy in, mat-vec, copy out on
+ * `stream`.  staging_dev: at least roundup(2*B*K, 1024) + 2*B*N bytes, 1024-byte aligned.
+ */
+int dq_decode_linear_host(const dq_weights *w, const void *X_host, int64_t B, int64_t ldx, void *Y_host,
+                          int64_t ldy, void *staging_dev, size_t staging_bytes, void *stream);
+
 /* ---- parity hooks: canonical encodings, compared bit for bit with the oracle ---- */
 
 /*

@@ -21,7 +21,8 @@ SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
            "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_export_canonical", "dq_import_canonical",
-           "dq_quantize_activations", "dq_get_status", "dq_weights_shape")
+           "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
+           "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
 
 class DQError(RuntimeError):
@@ -65,6 +66,12 @@ def lib() -> C.CDLL:
         L.dq_prefill_linear_static.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp]
         L.dq_decode_linear.restype = C.c_int
         L.dq_decode_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_prefill_host_staging_bytes.restype = C.c_int
+        L.dq_prefill_host_staging_bytes.argtypes = [vp, i64, C.POINTER(C.c_size_t)]
+        L.dq_prefill_linear_host.restype = C.c_int
+        L.dq_prefill_linear_host.argtypes = [vp, vp, i64, i64, C.c_float, vp, i64, vp, C.c_size_t, vp]
+        L.dq_decode_linear_host.restype = C.c_int
+        L.dq_decode_linear_host.argtypes = [vp, vp, i64, i64, vp, i64, vp, C.c_size_t, vp]
         L.dq_decode_linear_nvfp4.restype = C.c_int
         L.dq_decode_linear_nvfp4.argtypes = [vp, vp, i64, i64, vp, i64, vp]
         L.dq_import_canonical.restype = C.c_int
@@ -254,6 +261,33 @@ def decode_linear_nvfp4(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None,
     _check(lib().dq_decode_linear_nvfp4(w.handle, X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
                                         _stream_ptr(stream)), "dq_decode_linear_nvfp4")
     return out
+
+
+def prefill_host_staging_bytes(w: DQWeights, M: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().dq_prefill_host_staging_bytes(w.handle, M, C.byref(out)), "dq_prefill_host_staging_bytes")
+    return int(out.value)
+
+
+def prefill_linear_host(w: DQWeights, A_host: torch.Tensor, act_global_scale: float, Y_host: torch.Tensor,
+                        staging: torch.Tensor, stream=None) -> torch.Tensor:
+    """dq_prefill_linear_host: A_host / Y_host are (pinned) CPU tensors, staging a CUDA byte buffer."""
+    assert not A_host.is_cuda and not Y_host.is_cuda and staging.is_cuda
+    assert A_host.dtype == torch.bfloat16 and Y_host.dtype == torch.bfloat16 and A_host.stride(1) == 1
+    M = A_host.shape[0]
+    _check(lib().dq_prefill_linear_host(w.handle, A_host.data_ptr(), M, A_host.stride(0), float(act_global_scale),
+                                        Y_host.data_ptr(), Y_host.stride(0), staging.data_ptr(), staging.numel(),
+                                        _stream_ptr(stream)), "dq_prefill_linear_host")
+    return Y_host
+
+
+def decode_linear_host(w: DQWeights, X_host: torch.Tensor, Y_host: torch.Tensor, staging: torch.Tensor, stream=None):
+    """dq_decode_linear_host: X_host / Y_host are (pinned) CPU tensors, staging a CUDA byte buffer."""
+    assert not X_host.is_cuda and not Y_host.is_cuda and staging.is_cuda
+    _check(lib().dq_decode_linear_host(w.handle, X_host.data_ptr(), X_host.shape[0], X_host.stride(0),
+                                       Y_host.data_ptr(), Y_host.stride(0), staging.data_ptr(), staging.numel(),
+                                       _stream_ptr(stream)), "dq_decode_linear_host")
+    return Y_host
 
 
 def export_canonical(w: DQWeights, fmt: int, stream=None):

@@ -372,3 +372,30 @@ def test_calls_replay_from_a_cuda_graph(dq, oracle):
         assert torch.equal(got, want) and torch.equal(got_d, want_d)
     Yr, S = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A.cpu()), sa, ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
     check_outputs(_f64(Y), Yr, S, "graph replay prefill")
+
+
+def test_host_buffer_entry_points_match_device_calls(dq, oracle):
+    """Pinned host activations in, host outputs back, copies inside the call (row chunks pipelined over
+    three streams): same bits as the device-pointer calls; strided host rows; M not a multiple of a chunk."""
+    M, N, K = 2500, 512, 1024
+    W, _ = _layer(oracle, N, K, 80)
+    w = dq.pack_weights(W.to(DEV))
+    A_full = dq_inputs.gaussian_bf16(M, K + 64, 1.0, 81).pin_memory()
+    A_host = A_full[:, :K]
+    sa = dq_inputs.static_act_scale(A_host)
+    Y_full = torch.full((M, N + 32), 7.0, dtype=torch.bfloat16).pin_memory()
+    staging = dq.alloc_workspace(dq.prefill_host_staging_bytes(w, M), DEV)
+    for _ in range(2):                                   # twice in a row on the same stream
+        dq.prefill_linear_host(w, A_host, sa, Y_full[:, :N], staging)
+    torch.cuda.synchronize()
+    want = dq.prefill_linear(w, A_host.contiguous().to(DEV), sa)
+    _status_ok(dq)
+    assert torch.equal(Y_full[:, :N], want.cpu()) and torch.all(Y_full[:, N:] == 7.0)
+    X_host = A_host[:3]
+    Yd_host = torch.zeros(3, N, dtype=torch.bfloat16).pin_memory()
+    dq.decode_linear_host(w, X_host, Yd_host, staging)
+    torch.cuda.synchronize()
+    assert torch.equal(Yd_host, dq.decode_linear(w, X_host.contiguous().to(DEV)).cpu())
+    with pytest.raises(dq.DQError):
+        dq.prefill_linear_host(w, A_host, sa, Y_full[:, :N], staging[:4096])
+    _status_ok(dq)
