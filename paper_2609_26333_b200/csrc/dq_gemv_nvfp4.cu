@@ -55,6 +55,12 @@ __device__ __forceinline__ void ffma2(unsigned long long &acc, unsigned long lon
 {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 __device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
 {
     unsigned long long r;
@@ -180,29 +186,32 @@ gemv_nvfp4_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restrict__
             const uint32_t scw = r == 0 ? cur.sc.x : r == 1 ? cur.sc.y : r == 2 ? cur.sc.z : cur.sc.w;
             float d0, d1;
             e4m3x2_to_f32((widx & 1) ? (scw >> 16) : (scw & 0xFFFFu), d0, d1);
+            unsigned long long rowacc[BT];
 #pragma unroll
-            for (int t = 0; t < BT; ++t) v[r][t] = 0.0f;
+            for (int t = 0; t < BT; ++t) rowacc[t] = 0ull;
 #pragma unroll
             for (int blk = 0; blk < 2; ++blk) {
                 unsigned long long g[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const uint32_t word = cw[2 * blk + (q >> 2)];
-                    g[q] = ok ? lds_u64(__byte_perm(word, lane_base, 0x7604 | ((q & 3) << 4))) : 0ull;
+                    g[q] = lds_u64(__byte_perm(word, lane_base, 0x7604 | ((q & 3) << 4)));
                 }
+                const float d = blk ? d1 : d0;
+                const unsigned long long dd = pack_f32x2(d, d);
 #pragma unroll
                 for (int t = 0; t < BT; ++t) {
-                    unsigned long long acc0 = 0ull, acc1 = 0ull;
+                    unsigned long long acc = mul2(g[0], xs[t][8 * blk]);
 #pragma unroll
-                    for (int q = 0; q < 8; q += 2) {
-                        ffma2(acc0, g[q], xs[t][8 * blk + q]);
-                        ffma2(acc1, g[q + 1], xs[t][8 * blk + q + 1]);
-                    }
-                    float a0, a1, c0, c1;
-                    unpack_f32x2(acc0, a0, a1);
-                    unpack_f32x2(acc1, c0, c1);
-                    v[r][t] = fmaf(blk ? d1 : d0, (a0 + a1) + (c0 + c1), v[r][t]);
+                    for (int q = 1; q < 8; ++q) ffma2(acc, g[q], xs[t][8 * blk + q]);
+                    ffma2(rowacc[t], acc, dd);                    // block scale on both halves
                 }
+            }
+#pragma unroll
+            for (int t = 0; t < BT; ++t) {
+                float lo, hi;
+                unpack_f32x2(rowacc[t], lo, hi);
+                v[r][t] = lo + hi;
             }
         }
         // butterfly: afterwards lane l holds the warp total of row ((l>>4)&1)*2 + ((l>>3)&1)
