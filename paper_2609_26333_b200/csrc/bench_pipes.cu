@@ -118,6 +118,21 @@ template<int MODE> __global__ void __launch_bounds__(1024,1) k(uint32_t *out, lo
         r[4]^=a[0]^a[1]^a[2]^a[3];
         r[u]=shf(r[u],3);
       }
+    } else if (MODE==16){ // cvt e2m1x2 -> f16x2, x8
+      #pragma unroll
+      for(int i=0;i<8;i++){ uint32_t o; asm volatile("{.reg .b8 t; cvt.u8.u32 t, %1; cvt.rn.f16x2.e2m1x2 %0, t;}":"=r"(o):"r"(r[i])); r[i]=o; }
+    } else if (MODE==17){ // cvt e4m3x2 -> f16x2, x8
+      #pragma unroll
+      for(int i=0;i<8;i++){ uint32_t o; asm volatile("cvt.rn.f16x2.e4m3x2 %0, %1;":"=r"(o):"h"((unsigned short)r[i])); r[i]=o; }
+    } else if (MODE==18){ // NVFP4 weights to tensor cores: per 4 pairs 4 cvt e2m1x2 + 4 HMUL2 + 1 mma
+      #pragma unroll
+      for(int u=0;u<4;u++){
+        uint32_t a[4];
+        #pragma unroll
+        for(int i=0;i<4;i++){ uint32_t o; asm volatile("{.reg .b8 t; .reg .b32 w; shr.u32 w, %1, %2; cvt.u8.u32 t, w; cvt.rn.f16x2.e2m1x2 %0, t;}":"=r"(o):"r"(r[u]),"r"(8*i)); hmul2(a[i],o,seed); }
+        mma16816(d[u],a[0],a[1],a[2],a[3],r[4],r[5]);
+        r[u]=shf(r[u],3);
+      }
     } else if (MODE==13){ // HMUL2 x8
       #pragma unroll
       for(int i=0;i<8;i++) hmul2(r[i],r[i],seed);
@@ -146,7 +161,7 @@ template<int MODE> void run(const char*name,int ops_per_iter,int threads)
 int main(){
   for(int thr: {512,1024}){
     run<0>("PRMT",8,thr); run<1>("LOP3",8,thr); run<2>("SHF.wrap",8,thr); run<3>("LDS.32 dep",8,thr); run<4>("LDS.64 dep",8,thr);
-    run<5>("FFMA2",8,thr); run<6>("HFMA2",8,thr); run<13>("HMUL2",8,thr); run<8>("FFMA",8,thr); run<7>("mma.m16n8k16",4,thr);
+    run<5>("FFMA2",8,thr); run<6>("HFMA2",8,thr); run<13>("HMUL2",8,thr); run<16>("cvt f16x2.e2m1x2",8,thr); run<17>("cvt f16x2.e4m3x2",8,thr); run<18>("4 cvt.e2m1x2+4 HMUL2+1 mma [4 pairs]",4,thr); run<8>("FFMA",8,thr); run<7>("mma.m16n8k16",4,thr);
     run<9>("reg lookup + mma  [units: 4 pairs]",4,thr); run<14>("reg lookup only [4 pairs]",4,thr); run<10>("4 PRMT+4 LDS32+1 mma [4 pairs]",4,thr); run<15>("4 PRMT+4 LDS32 only [4 pairs]",4,thr);
     run<11>("4 PRMT+4 LDS64+4 FFMA2 [4 pairs]",4,thr); run<12>("half reg / half table + mma [4 pairs]",4,thr);
   }

@@ -379,6 +379,9 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
     return dq_prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream);
 }
 
+static int g_nv_decode_kernel = 1;      // 1 = tensor-core kernel, 0 = CUDA-core kernel (kept for comparison)
+int dq_debug_nvfp4_decode_kernel(int which) { int old = g_nv_decode_kernel; g_nv_decode_kernel = which; return old; }
+
 int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
                            void *stream)
 {
@@ -402,7 +405,9 @@ int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, in
     g.ldy = ldy;
     g.N = w->N;
     g.K = w->K;
-    if (dq::launch_gemv_nvfp4(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
+    const cudaError_t ce = g_nv_decode_kernel ? dq::launch_gemv_nvfp4_mma(g, reinterpret_cast<cudaStream_t>(stream))
+                                              : dq::launch_gemv_nvfp4(g, reinterpret_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
 

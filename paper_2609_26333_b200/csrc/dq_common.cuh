@@ -170,7 +170,8 @@ struct GemvNvArgs {
     void *Y; int64_t ldy;
     int64_t N, K;
 };
-cudaError_t launch_gemv_nvfp4(const GemvNvArgs &args, cudaStream_t stream);
+cudaError_t launch_gemv_nvfp4(const GemvNvArgs &args, cudaStream_t stream);          // CUDA cores, pair-table lookups
+cudaError_t launch_gemv_nvfp4_mma(const GemvNvArgs &args, cudaStream_t stream);      // tensor cores (mma.sync), no lookups
 cudaError_t launch_fill_e2m1_table(cudaStream_t stream);   // value-pair table of the NVFP4 decode kernel
 
 }  // namespace dq

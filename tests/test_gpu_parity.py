@@ -284,7 +284,7 @@ def test_decode_parity(dq, oracle, N, K, seed, B):
 
 
 @pytest.mark.parametrize("N,K,seed", [(512, 256, 0), (144, 384, 31), (784, 1152, 32), (272, 17408, 33)])
-@pytest.mark.parametrize("B", [1, 2, 3, 8])
+@pytest.mark.parametrize("B", [1, 2, 3, 8, 17, 64])
 def test_decode_nvfp4_parity(dq, oracle, N, K, seed, B):
     """Weight-only decode on the NVFP4 view; also from the LUT3-derived view of the same matrix."""
     W, ref = _layer(oracle, N, K, seed)
@@ -302,6 +302,27 @@ def test_decode_nvfp4_parity(dq, oracle, N, K, seed, B):
         w3 = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
         with pytest.raises(dq.DQError):
             dq.decode_linear_nvfp4(w3, X.to(DEV))
+
+
+def test_decode_nvfp4_kernels_agree_and_handle_wide_range_activations(dq, oracle):
+    """The tensor-core kernel (default) and the CUDA-core kernel both meet the oracle; activations spanning
+    many binades (the tensor-core kernel rescales them to fp16) and strided, guarded outputs."""
+    N, K, B = 400, 2048, 5
+    W, ref = _layer(oracle, N, K, 90)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    g = torch.Generator().manual_seed(91)
+    X = (torch.randn(B, K, generator=g) * torch.exp2(torch.randint(-20, 12, (B, K), generator=g).float())).to(torch.bfloat16)
+    Yr, S = oracle.decode_linear_nvfp4(dq_inputs.bf16_to_f32_numpy(X), ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
+    for which in (1, 0):
+        old = dq.lib().dq_debug_nvfp4_decode_kernel(which)
+        try:
+            out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+            dq.decode_linear_nvfp4(w, X.to(DEV), out=out[:, :N])
+            _status_ok(dq)
+        finally:
+            dq.lib().dq_debug_nvfp4_decode_kernel(old)
+        assert torch.all(out[:, N:] == -3.0)
+        check_outputs(_f64(out[:, :N]), Yr, S, f"nvfp4 decode kernel {which}, wide-range activations")
 
 
 def test_decode_one_hot_and_strided(dq, oracle):
