@@ -379,6 +379,8 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
     return dq_prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream);
 }
 
+static int g_lut_decode_kernel = -1;    // -1 = by batch size, 0 = CUDA-core kernel, 1 = tensor-core kernel
+int dq_debug_lut3_decode_kernel(int which) { int old = g_lut_decode_kernel; g_lut_decode_kernel = which; return old; }
 static int g_nv_decode_kernel = 1;      // 1 = tensor-core kernel, 0 = CUDA-core kernel (kept for comparison)
 int dq_debug_nvfp4_decode_kernel(int which) { int old = g_nv_decode_kernel; g_nv_decode_kernel = which; return old; }
 
@@ -434,7 +436,12 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
     g.ldy = ldy;
     g.N = w->N;
     g.K = w->K;
-    if (dq::launch_gemv_lut3(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
+    // batch 1: CUDA-core kernel; with two and more columns the tensor-core kernel wins (the batch rides along in
+    // the B operand: 17408x5120 at batch 2 / 8 / 16: 22 / 27 / 52 us against 26 / 103 / 206 us)
+    const bool use_mma = (g_lut_decode_kernel == 1) || (g_lut_decode_kernel < 0 && B >= 2);
+    const cudaError_t ce = use_mma ? dq::launch_gemv_lut3_mma(g, reinterpret_cast<cudaStream_t>(stream))
+                                   : dq::launch_gemv_lut3(g, reinterpret_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
 

@@ -160,7 +160,8 @@ struct GemvArgs {
     void *Y; int64_t ldy;
     int64_t N, K;
 };
-cudaError_t launch_gemv_lut3(const GemvArgs &args, cudaStream_t stream);
+cudaError_t launch_gemv_lut3(const GemvArgs &args, cudaStream_t stream);              // CUDA cores: batch 1 and 2
+cudaError_t launch_gemv_lut3_mma(const GemvArgs &args, cudaStream_t stream);          // tensor cores: eight columns per pass
 
 struct GemvNvArgs {
     const uint8_t *codes; const uint8_t *sf;              // NVFP4 view: [N][K/2] codes, MMA-layout scales

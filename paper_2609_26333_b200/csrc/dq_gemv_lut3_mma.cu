@@ -1,0 +1,362 @@
+// LUT3 decode for small batches with the products on tensor cores (App. C.2 kernel specification; the
+// skinny-batch case the paper leaves open, Sec. 5):
+//   Y[b][n] = bf16( s * sum_k d_blk(n,k) * G[idx(n,k)] * X[b][k] ),   up to eight batch columns per pass.
+// Same skeleton as the NVFP4 tensor-core decode kernel: a warp owns 16 consecutive rows and a 1024-weight
+// slice of K; lane (g, t) of the mma fragment layout holds rows g / g+8 and, per 512-weight half slice, four
+// consecutive plane words (128 weights) of each row; mma i contracts every lane's weights 4 i .. 4 i + 3.
+// Dequantisation: the three plane words are merged into bytes holding the six index bits of a weight pair
+// (two bitwise selects per four pairs after rotating the planes, as in the CUDA-core kernel), a byte addresses
+// a 64-entry table of fp16 level pairs in shared memory (one 4-byte slot per lane: conflict free).  The block
+// scale is applied in fp16 without loss: level * d is split into hi = rn(level * d) and lo = level * d - hi
+// (one multiply, one fused multiply-add; lo is exact), and both go through mma.sync.m16n8k16 with fp32
+// accumulation.  Activations: power-of-two scaling, fp16 in shared memory, one 8-byte load per pair of mmas.
+// At batch 1 this costs more instructions per weight than the CUDA-core kernel (which stays the batch-1
+// path, about 5 % faster there); from batch 2 on it wins because the batch rides along in the B operand.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "dq_common.cuh"
+#include "dq_tcgen05.cuh"
+
+namespace dq {
+
+namespace {
+
+constexpr int kSlots = 4;                         // cross-warp reduction slots per row group
+constexpr uint32_t kTableAddr = 0x4000;           // shared-window address of the level-pair table (16 KiB aligned)
+constexpr uint32_t kTableBytes = 16384;           // 64 entries x 256 B (first 128 B used: one 4-byte slot per lane)
+constexpr uint32_t kRedAddr = 0x8000;             // [G][kSlots][W][32 lanes][4] floats
+constexpr uint32_t kSmemLimit = 227 * 1024;       // the x columns follow the reduction buffers, up to this window address
+
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b)
+{
+    uint32_t r;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+// a * b - h on both halves (h = rn(a * b): the result is the exact rounding error of the product)
+__device__ __forceinline__ uint32_t hres2(uint32_t a, uint32_t b, uint32_t h)
+{
+    uint32_t r;
+    asm("{\n\t.reg .b32 n;\n\tneg.f16x2 n, %3;\n\tfma.rn.f16x2 %0, %1, %2, n;\n\t}" : "=r"(r) : "r"(a), "r"(b), "r"(h));
+    return r;
+}
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t rotr32(uint32_t x, int n) { return __funnelshift_r(x, x, n); }
+__device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t mask)      // mask ? a : b
+{
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(mask), "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t m, uint32_t o)          // (a & m) | o
+{
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(m), "r"(o));
+    return r;
+}
+
+// one 512-weight half slice of rows g / g+8: four plane words per plane and eight scale bytes per row
+struct HalfRegs { uint4 p[2][3]; uint2 sc[2]; };
+
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT, 1)
+gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
+                     const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
+                     __nv_bfloat16 *__restrict__ Y, int64_t ldy, int N, int K, int W, int G, uint32_t col_stride,
+                     uint32_t x_addr, StatusWord *status)
+{
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw);
+    volatile int *sync_words = reinterpret_cast<volatile int *>(smem_raw + 64);          // [G][kSlots] x (generation, count)
+    float *xmax_s = reinterpret_cast<float *>(smem_raw + 768);                          // 32 per-warp maxima
+    if (win0 + 1024 > kTableAddr) {
+        if (threadIdx.x == 0) { atomicExch(&status->status, (int)DQ_ERR_INTERNAL); atomicExch(&status->detail, 0x35000); }
+        return;
+    }
+    uint8_t *table = smem_raw + (kTableAddr - win0);
+    float *red = reinterpret_cast<float *>(smem_raw + (kRedAddr - win0));
+    uint8_t *xh = smem_raw + (x_addr - win0);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
+    const int grp = warp / W;
+    const int w = warp - grp * W;
+    const int g = lane >> 2, t = lane & 3;
+    const int slices = W;                                   // ceil(K / 1024)
+    const int kpad = slices * 1024;
+
+    if (threadIdx.x < 16 * kSlots * 2) sync_words[threadIdx.x] = 0;
+    if (threadIdx.x == 0) *abort_flag = 0;
+    // table: entry e (b0a b0b b1a b1b b2a b2b of a weight pair) -> half2(G[ia], G[ib]), one 4-byte slot per lane
+    for (int i = threadIdx.x; i < 64 * 32; i += blockDim.x) {
+        const int e = i >> 5, l = i & 31;
+        const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
+        const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
+        *reinterpret_cast<uint32_t *>(table + e * 256 + l * 4) = (hdr->lut_f16[ia] & 0xFFFFu) | (hdr->lut_f16[ib] << 16);
+    }
+
+    const int ntiles = N / 16;                              // N % 16 == 0
+    const int stride = gridDim.x * G;
+    const int first = blockIdx.x * G + grp;
+
+    auto load_half = [&](HalfRegs &R, int tile, int h) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int row = tile * 16 + g + 8 * half;
+            const uint8_t *blk = lut + ((size_t)row * slices + w) * kLutBlockBytes;
+#pragma unroll
+            for (int p = 0; p < 3; ++p)
+                R.p[half][p] = __ldg(reinterpret_cast<const uint4 *>(blk + p * 128 + h * 64 + t * 16));
+            R.sc[half] = __ldg(reinterpret_cast<const uint2 *>(blk + kLutScaleOff + h * 32 + t * 8));
+        }
+    };
+    // Register ring of two half slices: position p of the warp's stream is half p % 2 of tile first + (p / 2) * stride.
+    // The weights are constant data: start streaming before waiting for the kernel ahead of this one.
+    HalfRegs ring[2];
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            ring[p].sc[half] = make_uint2(0, 0);
+#pragma unroll
+            for (int q = 0; q < 3; ++q) ring[p].p[half][q] = make_uint4(0, 0, 0, 0);
+        }
+        if (first < ntiles) load_half(ring[p], first, p);
+    }
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ---- activations of this pass: largest magnitude -> power-of-two scale -> fp16 in shared memory
+    float m = 0.0f;
+    for (int c = 0; c < cols; ++c) {
+        const uint32_t *xp = reinterpret_cast<const uint32_t *>(X + (int64_t)(b0 + c) * ldx);
+        for (int i = threadIdx.x; i < K / 2; i += blockDim.x) {
+            const uint32_t v = __ldg(xp + i);
+            m = fmaxf(m, fmaxf(fabsf(__uint_as_float(v << 16)), fabsf(__uint_as_float(v & 0xFFFF0000u))));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) xmax_s[warp] = m;
+    __syncthreads();
+    m = 0.0f;
+    for (int i = 0; i < nwarps; ++i) m = fmaxf(m, xmax_s[i]);
+    int ex = (int)((__float_as_uint(m) >> 23) & 0xFFu) - 127;           // floor(log2(max)); -127 for zero / subnormal
+    ex = max(-100, min(100, ex));
+    const float xscale = __uint_as_float((uint32_t)(127 + 14 - ex) << 23);   // 2^(14 - ex)
+    const float xinv = __uint_as_float((uint32_t)(127 - 14 + ex) << 23);
+    for (int c = 0; c < cols; ++c) {
+        const uint4 *xp = reinterpret_cast<const uint4 *>(X + (int64_t)(b0 + c) * ldx);
+        for (int i = threadIdx.x; i < kpad / 8; i += blockDim.x) {
+            uint32_t r[4] = {0u, 0u, 0u, 0u};                       // the padding of a short last slice reads as zero
+            if (i < K / 8) {
+                const uint4 v = __ldg(xp + i);
+                const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                    const __half2 h = __floats2half2_rn(__uint_as_float(ww[z] << 16) * xscale,
+                                                        __uint_as_float(ww[z] & 0xFFFF0000u) * xscale);
+                    r[z] = *reinterpret_cast<const uint32_t *>(&h);
+                }
+            }
+            // Inside a 512-weight half slice lane t owns weights 128 t .. 128 t + 127; the four weights
+            // 128 t + 32 wi + 4 i .. + 3 (word wi, mma i of that word) sit at byte 256 wi + 32 i + 8 t, so that the
+            // B-fragment reads of one mma (lanes t, columns g 32 bytes apart mod 128) hit distinct banks.
+            const int k0 = i * 8;
+            const int hs = k0 >> 9, tt = (k0 >> 7) & 3, wi = (k0 >> 5) & 3, ii = (k0 & 31) >> 2;
+            uint8_t *dst = xh + (size_t)c * col_stride + (size_t)hs * 1024 + wi * 256 + ii * 32 + tt * 8;
+            *reinterpret_cast<uint2 *>(dst) = make_uint2(r[0], r[1]);
+            *reinterpret_cast<uint2 *>(dst + 32) = make_uint2(r[2], r[3]);
+        }
+    }
+    __syncthreads();
+    const float out_scale = hdr->s * xinv;
+    const uint32_t xlane = x_addr + (uint32_t)((g < cols) ? g : 0) * col_stride + (uint32_t)t * 8 + (uint32_t)w * 2048;
+    const uint32_t lane_base = kTableAddr | (uint32_t)(lane * 4);
+
+    bool ok = true;
+    int it = 0;
+    for (int tile = first; tile < ntiles; tile += stride, ++it) {
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            HalfRegs &cur = ring[h];
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi) {
+                uint32_t pw[2][3], dA[2], dB[2];
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const uint4 q0 = cur.p[half][0], q1 = cur.p[half][1], q2 = cur.p[half][2];
+                    pw[half][0] = wi == 0 ? q0.x : wi == 1 ? q0.y : wi == 2 ? q0.z : q0.w;
+                    pw[half][1] = wi == 0 ? q1.x : wi == 1 ? q1.y : wi == 2 ? q1.z : q1.w;
+                    pw[half][2] = wi == 0 ? q2.x : wi == 1 ? q2.y : wi == 2 ? q2.z : q2.w;
+                    const uint32_t scw = (wi < 2) ? (cur.sc[half].x >> (16 * wi)) : (cur.sc[half].y >> (16 * (wi - 2)));
+                    uint32_t d2;
+                    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(d2) : "h"((unsigned short)scw));
+                    dA[half] = __byte_perm(d2, d2, 0x1010);          // first block of the word on both halves
+                    dB[half] = __byte_perm(d2, d2, 0x3232);          // second block
+                }
+                const uint32_t xa = xlane + (uint32_t)h * 1024 + (uint32_t)wi * 256;
+#pragma unroll
+                for (int gg = 0; gg < 4; ++gg) {                     // pairs 4 gg .. 4 gg + 3: mmas 2 gg and 2 gg + 1
+                    uint32_t u[2];
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const uint32_t a = gg ? rotr32(pw[half][0], 2 * gg) : pw[half][0];
+                        const uint32_t b = gg ? rotr32(pw[half][1], 2 * gg) : pw[half][1];
+                        const uint32_t c = gg ? rotr32(pw[half][2], 2 * gg) : pw[half][2];
+                        // byte j: bits 0-1 plane 0, 2-3 plane 1, 4-5 plane 2 of pair 4 gg + j; bit 6 selects the table
+                        u[half] = and_or(bitsel(bitsel(a, b, 0x03030303u), c, 0x0F0F0F0Fu), 0x3F3F3F3Fu, 0x40404040u);
+                    }
+                    const uint32_t d0 = (gg < 2) ? dA[0] : dB[0], d1 = (gg < 2) ? dA[1] : dB[1];
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const uint32_t v0 = lds_u32(__byte_perm(u[0], lane_base, 0x7604 | ((2 * jj) << 4)));      // row g, pair 2 mm
+                        const uint32_t v2 = lds_u32(__byte_perm(u[0], lane_base, 0x7604 | ((2 * jj + 1) << 4)));  // row g, pair 2 mm + 1
+                        const uint32_t v1 = lds_u32(__byte_perm(u[1], lane_base, 0x7604 | ((2 * jj) << 4)));      // row g + 8
+                        const uint32_t v3 = lds_u32(__byte_perm(u[1], lane_base, 0x7604 | ((2 * jj + 1) << 4)));
+                        const uint32_t h0 = hmul2(v0, d0), h1 = hmul2(v1, d1), h2 = hmul2(v2, d0), h3 = hmul2(v3, d1);
+                        const uint2 xv = lds_v2(xa + (uint32_t)(2 * gg + jj) * 32);
+                        mma16816(acc, h0, h1, h2, h3, xv.x, xv.y);
+                        mma16816(acc, hres2(v0, d0, h0), hres2(v1, d1, h1), hres2(v2, d0, h2), hres2(v3, d1, h3), xv.x, xv.y);
+                    }
+                }
+            }
+            // the slot is consumed: refill it with the same half of the warp's next tile (the other half
+            // slice, loaded one step earlier, is what the warp works on meanwhile)
+            if (tile + stride < ntiles) load_half(cur, tile + stride, h);
+        }
+        // ---- cross-warp sum: last-arriving warp of the group adds the W partial fragments in order and stores
+        const int slot = it & (kSlots - 1);
+        volatile int *gen = sync_words + (grp * kSlots + slot) * 2;
+        int *cnt = const_cast<int *>(gen) + 1;
+        if (ok) {
+            uint32_t good = 1;
+            if (lane == 0) {
+                const int want = it / kSlots;
+                long long t0 = 0;
+                uint32_t spins = 0;
+                while (*gen != want) {
+                    if ((++spins & 255u) == 0u) {
+                        if (t0 == 0) t0 = clock64();
+                        if (*abort_flag || clock64() - t0 > tc::kWaitBudgetCycles) { *abort_flag = 1; good = 0; break; }
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+        }
+        float4 *rbuf = reinterpret_cast<float4 *>(red) + (size_t)((grp * kSlots + slot) * W) * 32;
+        rbuf[w * 32 + lane] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        __syncwarp();
+        int prev = 0;
+        if (lane == 0) { __threadfence_block(); prev = atomicAdd(cnt, 1); }
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev == W - 1) {
+            __threadfence_block();
+            float tot[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            for (int ww = 0; ww < W; ++ww) {
+                const volatile float *p = reinterpret_cast<const volatile float *>(rbuf + ww * 32 + lane);
+                tot[0] += p[0]; tot[1] += p[1]; tot[2] += p[2]; tot[3] += p[3];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {                    // c0, c1: row g, columns 2t, 2t+1; c2, c3: row g + 8
+                const int col = 2 * t + (j & 1);
+                const int row = tile * 16 + g + 8 * (j >> 1);
+                if (ok && col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot[j] * out_scale);
+            }
+            __syncwarp();
+            if (lane == 0) { *cnt = 0; __threadfence_block(); *gen = it / kSlots + 1; }
+        }
+    }
+    if (*abort_flag && lane == 0) {
+        atomicExch(&status->status, (int)DQ_ERR_TIMEOUT);
+        atomicExch(&status->detail, 0x36000 | (int)blockIdx.x);
+    }
+}
+
+template <int MAXT>
+cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int threads, int W, int G, uint32_t col_stride,
+                       uint32_t x_addr, uint32_t smem, cudaStream_t stream)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut3_mma_kernel<MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_lut3_mma_kernel<MAXT>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
+                              (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
+                              (int)a.K, W, G, col_stride, x_addr, a.status);
+}
+
+}  // namespace
+
+// batches of two and more: up to eight columns per pass on tensor cores
+cudaError_t launch_gemv_lut3_mma(const GemvArgs &a, cudaStream_t stream)
+{
+    const int K = (int)a.K, N = (int)a.N, B = (int)a.B;
+    const int W = (K + 1023) / 1024;                  // warps per row group (one 1024-weight slice each)
+    if (W > 32) return cudaErrorInvalidValue;
+    const int max_warps = (W > 20) ? 32 : 20;
+    int G = max_warps / W;
+    if (G < 1) G = 1;
+    if (G > 15) G = 15;
+    const int threads = G * W * 32;
+    const uint32_t red_bytes = (uint32_t)G * kSlots * W * 32 * 16;
+    const uint32_t x_addr = kRedAddr + ((red_bytes + 1023u) & ~1023u);
+    const uint32_t col_stride = (uint32_t)W * 2048u + 32u;       // padded K in fp16, 32 mod 128 (see the layout note)
+    int cols_max = (int)((kSmemLimit - 2048u - x_addr) / col_stride);
+    if (cols_max > 8) cols_max = 8;
+    if (cols_max < 1) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int ntiles = N / 16;
+    int grid = (ntiles + G - 1) / G;
+    if (grid > sms) grid = sms;
+    for (int b0 = 0; b0 < B; b0 += cols_max) {
+        const int cols = (B - b0 < cols_max) ? (B - b0) : cols_max;
+        const uint32_t smem = x_addr + (uint32_t)cols * col_stride;
+        cudaError_t e = (threads <= 512)   ? launch_one<512>(a, b0, cols, grid, threads, W, G, col_stride, x_addr, smem, stream)
+                        : (threads <= 640) ? launch_one<640>(a, b0, cols, grid, threads, W, G, col_stride, x_addr, smem, stream)
+                                           : launch_one<1024>(a, b0, cols, grid, threads, W, G, col_stride, x_addr, smem, stream);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace dq

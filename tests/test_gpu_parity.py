@@ -325,6 +325,25 @@ def test_decode_nvfp4_kernels_agree_and_handle_wide_range_activations(dq, oracle
         check_outputs(_f64(out[:, :N]), Yr, S, f"nvfp4 decode kernel {which}, wide-range activations")
 
 
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(272, 17408, 33)])
+@pytest.mark.parametrize("B", [1, 3, 8, 11])
+def test_decode_lut3_tensor_core_kernel_parity(dq, oracle, N, K, seed, B):
+    """The tensor-core LUT3 kernel (the batch >= 3 path), forced for every batch size here."""
+    W, ref = _layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    X = dq_inputs.gaussian_bf16(B, K, 1.0, 2000 + seed + B)
+    old = dq.lib().dq_debug_lut3_decode_kernel(1)
+    try:
+        out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+        dq.decode_linear(w, X.to(DEV), out=out[:, :N])
+        _status_ok(dq)
+    finally:
+        dq.lib().dq_debug_lut3_decode_kernel(old)
+    assert torch.all(out[:, N:] == -3.0)
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 tensor-core decode {B}x{N}x{K}")
+
+
 def test_decode_one_hot_and_strided(dq, oracle):
     N, K = 256, 512
     W, ref = _layer(oracle, N, K, 64)
