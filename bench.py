@@ -37,8 +37,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum);
 # see profiles/ for the captures these come from.  None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {
-    ("gemm", "c3_gate_up27b"): 221.4e6 + 235.2e6,     # profiles/launch_list_c3_gate_up27b.md
-    ("gemv", "c3_gate_up27b"): 39.04e6,
+    ("gemm", "c3_gate_up27b"): 79.2e6 + 240.4e6,      # profiles/launch_list_c3_gate_up27b.md
+    ("gemv", "c3_gate_up27b"): 39.10e6,
 }
 
 
