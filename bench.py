@@ -135,8 +135,8 @@ def run_reference(args, cfg):
         return
     import oracle
     oracle.build()
-    # rows per step: about 0.9 s of oracle work, so that the default 200 steps end within minutes
-    rows = args.ref_rows or max(16, min(cfg.M, int(0.9 * 0.05e12 / (2.0 * cfg.N * cfg.K)) // 16 * 16))
+    # rows per step: about half a second of oracle work, so that the default 200 steps end within minutes
+    rows = args.ref_rows or max(16, min(cfg.M, int(0.5 * 0.05e12 / (2.0 * cfg.N * cfg.K)) // 16 * 16))
     W = dq_inputs.make_weight(cfg)
     W_f32 = dq_inputs.bf16_to_f32_numpy(W)
     A = dq_inputs.make_activations(cfg, rows)
