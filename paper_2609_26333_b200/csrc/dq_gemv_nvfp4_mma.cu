@@ -137,10 +137,14 @@ gemv_nvfp4_mma_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restri
     // ---- activations of this pass: largest magnitude -> power-of-two scale -> fp16 in shared memory
     float m = 0.0f;
     for (int c = 0; c < cols; ++c) {
-        const uint32_t *xp = reinterpret_cast<const uint32_t *>(X + (int64_t)(b0 + c) * ldx);
-        for (int i = threadIdx.x; i < K / 2; i += blockDim.x) {
-            const uint32_t v = __ldg(xp + i);
-            m = fmaxf(m, fmaxf(fabsf(__uint_as_float(v << 16)), fabsf(__uint_as_float(v & 0xFFFF0000u))));
+        const uint4 *xp = reinterpret_cast<const uint4 *>(X + (int64_t)(b0 + c) * ldx);
+        for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
+            const uint4 v = __ldg(xp + i);
+            // |bf16| pairs compare like unsigned integers once the sign bits are cleared
+            const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+            const uint32_t hi = max(max(a0 >> 16, a1 >> 16), max(a2 >> 16, a3 >> 16));
+            const uint32_t lo = max(max(a0 & 0xFFFFu, a1 & 0xFFFFu), max(a2 & 0xFFFFu, a3 & 0xFFFFu));
+            m = fmaxf(m, __uint_as_float(max(hi, lo) << 16));
         }
     }
 #pragma unroll
