@@ -39,6 +39,7 @@ L2_BYTES = 126 * 1024 * 1024
 NCU_TRAFFIC_BYTES = {
     ("gemm", "c3_gate_up27b"): 79.2e6 + 240.4e6,      # profiles/launch_list_c3_gate_up27b.md
     ("gemv", "c3_gate_up27b"): 39.10e6,
+    ("gemv_nvfp4", "c3_gate_up27b"): 50.2e6,          # profiles/gemv_nvfp4_mma_8192x4096.md (scaled by N x K)
 }
 
 
@@ -514,6 +515,14 @@ def main():
                             "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)),
                             "peak_source": f"{peaks['source']} copy bandwidth"},
     }
+    nv_bytes = 0.5625 * N * K + 2.0 * B * (K + N)
+    line["roofline_decode_nvfp4a16"] = {"kernel": "gemv_nvfp4_mma_kernel", "bound": "hbm",
+                                        "achieved": nv_bytes / (d_nv_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                        "frac": nv_bytes / (d_nv_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                        "traffic": NCU_TRAFFIC_BYTES.get(("gemv_nvfp4", cfg.name)),
+                                        "timing": "back-to-back launches", "peak_source": f"{peaks['source']} copy bandwidth"}
+    line["roofline_decode"]["back_to_back"] = {"achieved": dec_bytes / (d_b2b_ms * 1e-3) / 1e9,
+                                               "frac": dec_bytes / (d_b2b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     if e2e:
         line["e2e"] = {"value": world * flops / (e2e_p_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": int(2 * M * K + 2 * B * K), "d2h_bytes_per_step": int(2 * M * N + 2 * B * N),
