@@ -34,14 +34,14 @@ constexpr size_t kLutTableBytes = 65536;   // 256 entries x 32 lane slots x (fp3
 
 // LUT3 device layout: the weights of one row are cut into slices of 1024 (one per warp of the
 // decode kernel); slice s of row r is one block of 448 bytes:
-//   [plane 0: 32 words][plane 1: 32 words][plane 2: 32 words][scales: 64 signed E4M3 bytes]
-// i.e. 3 bit-plane words + 2 scale bytes per lane, 3.5 bit per weight.  A partial last slice is
+//   [word 0 of 32 triplets][word 1 of 32 triplets][word 2 of 32 triplets][scales: 64 signed E4M3 bytes]
+// i.e. 3 index words + 2 scale bytes per 32 weights, 3.5 bit per weight (bit order: lut3_locate below).  A partial last slice is
 // zero padded (zero scales, so the padding contributes nothing).
 constexpr int kLutSlice = 1024;
 constexpr int kLutBlockBytes = 448;
 constexpr int kLutScaleOff = 384;
 __host__ __device__ inline int64_t lut_slices(int64_t K) { return (K + kLutSlice - 1) / kLutSlice; }
-// word j (32 weights) of plane p in row r; K/32 words per row
+// word p (0..2) of triplet j (32 weights) in row r; K/32 triplets per row
 __host__ __device__ inline size_t lut_word_offset(int64_t r, int64_t j, int p, int64_t K)
 {
     return (size_t)(r * lut_slices(K) + j / 32) * kLutBlockBytes + (size_t)p * 128 + (size_t)(j % 32) * 4;
@@ -95,16 +95,24 @@ __host__ __device__ inline size_t sf_swizzled_offset(int64_t r, int64_t b, int64
     return (size_t)atom * 512 + (size_t)(rr % 32) * 16 + (size_t)(rr / 32) * 4 + (size_t)(b % 4);
 }
 
-// LUT3 device bit order.  The planes keep the (N, 3, K/32) int32 shape of App. C.2; inside a
-// word the 32 weights are permuted so that the decode kernel can assemble the six index bits of
-// two neighbouring weights (2q, 2q+1) into one byte with two bitwise selects:
-//   q = 4g + j  ->  plane p holds bit p of weight 2q+e at position (8j + 2g + e + 2p) mod 32.
-// Rotating the three plane words right by 2g and taking bits {0,1} / {2,3} / {4,5} of byte j from
-// planes 0 / 1 / 2 yields  b0a b0b b1a b1b b2a b2b  in the low six bits of that byte.
-__host__ __device__ inline int lut3_bitpos(int plane, int i)
+// LUT3 device bit order.  Storage stays three 32-bit words per 32 weights (3 bit per weight), in the three
+// 128-byte "plane" regions of a block, but the words are not bit-planes: words 0, 1, 2 hold the indices of
+// weights 0-7, 8-15, 16-23 as nibbles (weight 8a + n in bits 4n .. 4n+2 of word a), and the spare top bit of
+// the eight nibbles of word b holds bit b of the indices of weights 24-31 (weight 24 + n in bit 4n + 3).
+// A decode kernel gets byte-permute selectors / pair indices for 24 weights with one AND per word and for the
+// last eight with three shifts and three bitwise ops.  The canonical (export) layout is the bit-plane form.
+__host__ __device__ inline void lut3_locate(int bit, int i, int &word, int &pos)
 {
-    const int q = i >> 1, e = i & 1;
-    return (8 * (q & 3) + 2 * (q >> 2) + e + 2 * plane) & 31;
+    if (i < 24) { word = i >> 3; pos = 4 * (i & 7) + bit; }
+    else { word = bit; pos = 4 * (i - 24) + 3; }
+}
+// the four selector words of a word triplet: nibble n of word a is the index of weight 8a + n
+__device__ __forceinline__ void lut3_selectors(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t (&sel)[4])
+{
+    sel[0] = w0 & 0x77777777u;
+    sel[1] = w1 & 0x77777777u;
+    sel[2] = w2 & 0x77777777u;
+    sel[3] = ((w0 >> 3) & 0x11111111u) | ((w1 >> 2) & 0x22222222u) | ((w2 >> 1) & 0x44444444u);
 }
 
 // Device status word: [0] = dq_status, [1] = detail.

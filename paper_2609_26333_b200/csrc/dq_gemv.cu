@@ -1,32 +1,26 @@
-// LUT3 weight-only decode mat-vec / skinny GEMM (App. C.2 "Kernel specification"):
+// LUT3 weight-only decode mat-vec (App. C.2 "Kernel specification"), the batch-1 path:
 //   Y[b][n] = bf16( s * sum_blk d_blk * sum_{k in blk} G[idx(n,k)] * X[b][k] )
-// Weights stream from HBM as 3 bit-planes + one signed E4M3 scale per 16 weights
-// (3.5 bit per weight); they are dequantised in registers and accumulated in fp32
-// on the plain ALUs.
+// Weights stream from HBM as three index words per 32 weights + one signed E4M3 scale per 16 weights
+// (3.5 bit per weight); they are dequantised in registers and accumulated in fp32 on the plain ALUs.
 //
-// Work split.  K is cut into slices of 1024 weights; warp w of a row group owns
-// slice w for every row, lane l owns the 32 weights of plane word 32 w + l.  A
-// lane therefore keeps its 32 activations in registers (as fp32 pairs) for the
-// whole kernel and reads, per row, one coalesced 32-bit word of each plane and
-// two scale bytes, all at fixed offsets inside the 448-byte block of its slice.  Rows are taken four at a time with the next four already in
-// flight (two register buffers).  Partial sums meet in a warp butterfly, then across the warps
-// of the group through shared memory.
+// Work split.  K is cut into slices of 1024 weights; warp w of a row group owns slice w for every row,
+// lane l owns the 32 weights of word triplet 32 w + l.  A lane therefore keeps its 32 activations in
+// registers (as fp32 pairs) for the whole kernel and reads, per row, one 32-bit word of each of the three
+// word regions and two scale bytes, all at fixed offsets inside the 448-byte block of its slice.  Four rows
+// of all slices are contiguous in memory and arrive with one bulk copy into a shared-memory ring.  Partial
+// sums meet in a warp butterfly, then across the warps of the group through shared memory.
 //
-// Dequantisation.  Two bitwise selects merge the three plane words into a word
-// whose bytes each hold the six index bits of two neighbouring weights (see
-// lut3_bitpos); one byte-permute turns such a byte into the shared-memory
-// address of a 256-entry table of level pairs (the fp16 codebook widened to fp32;
-// entry stride 256 B, one 8-byte slot per lane, so lookups never collide on a
-// bank); the pair is multiplied into the accumulator pair with one packed fp32
-// FMA.  (Looking up fp16 pairs and widening them in registers halves the
-// shared-memory traffic but the conversion runs on the quarter-rate XU pipe,
-// which then limits the kernel: measured 14 weights/clk/SM.)
+// Dequantisation.  The device bit order (lut3_locate) stores indices as nibbles, so one AND per word (three
+// shifts and three bitwise ops for the last eight weights) gives selector words whose bytes each hold the
+// indices of two neighbouring weights; one byte-permute turns such a byte into the shared-memory address of a
+// table of level pairs (the fp16 codebook widened to fp32; entry stride 256 B, one 8-byte slot per lane, so
+// lookups never collide on a bank); the pair is multiplied into the accumulator pair with one packed fp32 FMA.
+// (Looking up fp16 pairs and widening them in registers halves the shared-memory traffic but costs two more
+// instructions per pair: measured 14 weights/clk/SM.)
 //
-// What bounds it.  Per weight the kernel needs about 1 bit-manipulation
-// instruction, half a 64-bit shared-memory lookup and half a packed FMA; on B200
-// that is 16 weights/clk/SM (about 2 TB/s of weight traffic), set by the
-// shared-memory lookups and instruction issue, not by HBM.  The streaming
-// skeleton alone (ring, plane reads, reduction, no lookups) runs at 4.1 TB/s.
+// What bounds it.  One 64-bit shared-memory lookup per weight pair caps this formulation at 32 weights per
+// clock per SM; the kernel reaches 16-18 (about 2 TB/s of weight traffic), HBM would deliver 52.  The
+// streaming skeleton alone (ring, word reads, reduction, no lookups) runs at 4.1 TB/s.
 #include "dq_common.cuh"
 #include "dq_tcgen05.cuh"
 
@@ -60,14 +54,6 @@ __device__ __forceinline__ unsigned long long lds_u64(uint32_t addr)
     unsigned long long v;
     asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr));
     return v;
-}
-__device__ __forceinline__ uint32_t rotr32(uint32_t x, int n) { return __funnelshift_r(x, x, n); }
-// bits where mask is set come from a, the others from b
-__device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t mask)
-{
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(mask), "r"(a), "r"(b));   // mask ? a : b
-    return r;
 }
 // packed fp32 pair FMA: acc += a * b on both halves
 __device__ __forceinline__ void ffma2(unsigned long long &acc, unsigned long long a, unsigned long long b)
@@ -118,25 +104,24 @@ __device__ __forceinline__ void dot32_rows(const uint32_t (&p0)[R], const uint32
                                            const unsigned long long (&xs)[BT][16], float (&out)[R][BT])
 {
     float d[R][2];
+    uint32_t sel[R][4];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
+        lut3_selectors(p0[r], p1[r], p2[r], sel[r]);
         e4m3x2_to_f32(sc[r], d[r][0], d[r][1]);
 #pragma unroll
         for (int t = 0; t < BT; ++t) out[r][t] = 0.0f;
     }
 #pragma unroll
-    for (int blk = 0; blk < 2; ++blk) {          // pairs 0..7 are block 0 (rotations 0, 2), pairs 8..15 block 1
+    for (int blk = 0; blk < 2; ++blk) {          // pairs 0..7 are block 0, pairs 8..15 block 1
         unsigned long long gp[R][8];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int g = 2 * blk + h;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const uint32_t a = g ? rotr32(p0[r], 2 * g) : p0[r];
-                const uint32_t b = g ? rotr32(p1[r], 2 * g) : p1[r];
-                const uint32_t c = g ? rotr32(p2[r], 2 * g) : p2[r];
-                // byte j: bits 0-1 from plane 0, 2-3 from plane 1, 4-5 from plane 2 (6-7: other weights' bits)
-                const uint32_t u = bitsel(bitsel(a, b, 0x03030303u), c, 0x0F0F0F0Fu);
+                // selector word g: byte j holds the indices of weight pair 4g + j as nibbles (idx_b << 4 | idx_a)
+                const uint32_t u = sel[r][g];
 #pragma unroll
                 for (int j = 0; j < 4; ++j)      // address = table base | byte j of u << 8 | lane * 8
                     gp[r][4 * h + j] = lds_u64(__byte_perm(u, lane_base, 0x7604 | (j << 4)));

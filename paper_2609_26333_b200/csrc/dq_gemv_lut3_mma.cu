@@ -4,9 +4,9 @@
 // Same skeleton as the NVFP4 tensor-core decode kernel: a warp owns 16 consecutive rows and a 1024-weight
 // slice of K; lane (g, t) of the mma fragment layout holds rows g / g+8 and, per 512-weight half slice, four
 // consecutive plane words (128 weights) of each row; mma i contracts every lane's weights 4 i .. 4 i + 3.
-// Dequantisation: the three plane words are merged into bytes holding the six index bits of a weight pair
-// (two bitwise selects per four pairs after rotating the planes, as in the CUDA-core kernel), a byte addresses
-// a 64-entry table of fp16 level pairs in shared memory (one 4-byte slot per lane: conflict free).  The block
+// Dequantisation without shared memory: the device bit order stores indices as nibbles, which are the
+// selectors of byte-permute; the eight fp16 levels live in four registers (low bytes, high bytes), two
+// permutes look up the bytes of four weights and two more interleave them into two fp16 pairs.  The block
 // scale is applied in fp16 without loss: level * d is split into hi = rn(level * d) and lo = level * d - hi
 // (one multiply, one fused multiply-add; lo is exact), and both go through mma.sync.m16n8k16 with fp32
 // accumulation.  Activations: power-of-two scaling, fp16 in shared memory, one 8-byte load per pair of mmas.
@@ -23,9 +23,7 @@ namespace dq {
 namespace {
 
 constexpr int kSlots = 4;                         // cross-warp reduction slots per row group
-constexpr uint32_t kTableAddr = 0x4000;           // shared-window address of the level-pair table (16 KiB aligned)
-constexpr uint32_t kTableBytes = 16384;           // 64 entries x 256 B (first 128 B used: one 4-byte slot per lane)
-constexpr uint32_t kRedAddr = 0x8000;             // [G][kSlots][W][32 lanes][4] floats
+constexpr uint32_t kRedAddr = 0x1000;             // shared-window address of [G][kSlots][W][32 lanes][4] floats
 constexpr uint32_t kSmemLimit = 227 * 1024;       // the x columns follow the reduction buffers, up to this window address
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -55,25 +53,6 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr)
     asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t rotr32(uint32_t x, int n) { return __funnelshift_r(x, x, n); }
-__device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t mask)      // mask ? a : b
-{
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(mask), "r"(a), "r"(b));
-    return r;
-}
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t m, uint32_t o)          // (a & m) | o
-{
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(m), "r"(o));
-    return r;
-}
 
 // one 512-weight half slice of rows g / g+8: four plane words per plane and eight scale bytes per row
 struct HalfRegs { uint4 p[2][3]; uint2 sc[2]; };
@@ -90,11 +69,10 @@ gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw);
     volatile int *sync_words = reinterpret_cast<volatile int *>(smem_raw + 64);          // [G][kSlots] x (generation, count)
     float *xmax_s = reinterpret_cast<float *>(smem_raw + 768);                          // 32 per-warp maxima
-    if (win0 + 1024 > kTableAddr) {
+    if (win0 + 1024 > kRedAddr) {
         if (threadIdx.x == 0) { atomicExch(&status->status, (int)DQ_ERR_INTERNAL); atomicExch(&status->detail, 0x35000); }
         return;
     }
-    uint8_t *table = smem_raw + (kTableAddr - win0);
     float *red = reinterpret_cast<float *>(smem_raw + (kRedAddr - win0));
     uint8_t *xh = smem_raw + (x_addr - win0);
 
@@ -109,12 +87,14 @@ gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
 
     if (threadIdx.x < 16 * kSlots * 2) sync_words[threadIdx.x] = 0;
     if (threadIdx.x == 0) *abort_flag = 0;
-    // table: entry e (b0a b0b b1a b1b b2a b2b of a weight pair) -> half2(G[ia], G[ib]), one 4-byte slot per lane
-    for (int i = threadIdx.x; i < 64 * 32; i += blockDim.x) {
-        const int e = i >> 5, l = i & 31;
-        const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
-        const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
-        *reinterpret_cast<uint32_t *>(table + e * 256 + l * 4) = (hdr->lut_f16[ia] & 0xFFFFu) | (hdr->lut_f16[ib] << 16);
+    // the eight fp16 levels as byte-permute tables: low bytes of levels 0-3 / 4-7, high bytes of levels 0-3 / 4-7
+    uint32_t tl0 = 0, tl1 = 0, th0 = 0, th1 = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        tl0 |= (hdr->lut_f16[j] & 0xFFu) << (8 * j);
+        th0 |= ((hdr->lut_f16[j] >> 8) & 0xFFu) << (8 * j);
+        tl1 |= (hdr->lut_f16[4 + j] & 0xFFu) << (8 * j);
+        th1 |= ((hdr->lut_f16[4 + j] >> 8) & 0xFFu) << (8 * j);
     }
 
     const int ntiles = N / 16;                              // N % 16 == 0
@@ -199,7 +179,6 @@ gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     __syncthreads();
     const float out_scale = hdr->s * xinv;
     const uint32_t xlane = x_addr + (uint32_t)((g < cols) ? g : 0) * col_stride + (uint32_t)t * 8 + (uint32_t)w * 2048;
-    const uint32_t lane_base = kTableAddr | (uint32_t)(lane * 4);
 
     bool ok = true;
     int it = 0;
@@ -224,24 +203,20 @@ gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
                     dB[half] = __byte_perm(d2, d2, 0x3232);          // second block
                 }
                 const uint32_t xa = xlane + (uint32_t)h * 1024 + (uint32_t)wi * 256;
+                uint32_t sel[2][4];
+                lut3_selectors(pw[0][0], pw[0][1], pw[0][2], sel[0]);
+                lut3_selectors(pw[1][0], pw[1][1], pw[1][2], sel[1]);
 #pragma unroll
-                for (int gg = 0; gg < 4; ++gg) {                     // pairs 4 gg .. 4 gg + 3: mmas 2 gg and 2 gg + 1
-                    uint32_t u[2];
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const uint32_t a = gg ? rotr32(pw[half][0], 2 * gg) : pw[half][0];
-                        const uint32_t b = gg ? rotr32(pw[half][1], 2 * gg) : pw[half][1];
-                        const uint32_t c = gg ? rotr32(pw[half][2], 2 * gg) : pw[half][2];
-                        // byte j: bits 0-1 plane 0, 2-3 plane 1, 4-5 plane 2 of pair 4 gg + j; bit 6 selects the table
-                        u[half] = and_or(bitsel(bitsel(a, b, 0x03030303u), c, 0x0F0F0F0Fu), 0x3F3F3F3Fu, 0x40404040u);
-                    }
+                for (int gg = 0; gg < 4; ++gg) {                     // weights 8 gg .. 8 gg + 7: mmas 2 gg and 2 gg + 1
                     const uint32_t d0 = (gg < 2) ? dA[0] : dB[0], d1 = (gg < 2) ? dA[1] : dB[1];
 #pragma unroll
-                    for (int jj = 0; jj < 2; ++jj) {
-                        const uint32_t v0 = lds_u32(__byte_perm(u[0], lane_base, 0x7604 | ((2 * jj) << 4)));      // row g, pair 2 mm
-                        const uint32_t v2 = lds_u32(__byte_perm(u[0], lane_base, 0x7604 | ((2 * jj + 1) << 4)));  // row g, pair 2 mm + 1
-                        const uint32_t v1 = lds_u32(__byte_perm(u[1], lane_base, 0x7604 | ((2 * jj) << 4)));      // row g + 8
-                        const uint32_t v3 = lds_u32(__byte_perm(u[1], lane_base, 0x7604 | ((2 * jj + 1) << 4)));
+                    for (int jj = 0; jj < 2; ++jj) {                 // four weights (two pairs) of each row per mma
+                        const uint32_t s0 = jj ? (sel[0][gg] >> 16) : sel[0][gg];
+                        const uint32_t s1 = jj ? (sel[1][gg] >> 16) : sel[1][gg];
+                        const uint32_t lo0 = __byte_perm(tl0, tl1, s0), hi0 = __byte_perm(th0, th1, s0);   // row g
+                        const uint32_t lo1 = __byte_perm(tl0, tl1, s1), hi1 = __byte_perm(th0, th1, s1);   // row g + 8
+                        const uint32_t v0 = __byte_perm(lo0, hi0, 0x5140), v2 = __byte_perm(lo0, hi0, 0x7362);
+                        const uint32_t v1 = __byte_perm(lo1, hi1, 0x5140), v3 = __byte_perm(lo1, hi1, 0x7362);
                         const uint32_t h0 = hmul2(v0, d0), h1 = hmul2(v1, d1), h2 = hmul2(v2, d0), h3 = hmul2(v3, d1);
                         const uint2 xv = lds_v2(xa + (uint32_t)(2 * gg + jj) * 32);
                         mma16816(acc, h0, h1, h2, h3, xv.x, xv.y);

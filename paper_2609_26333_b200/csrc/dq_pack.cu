@@ -195,16 +195,15 @@ cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, 
 
 // ------------------------------------------------------- decode pair table
 
-// Image of the decode kernel's shared-memory table, built once at pack time: entry e (a byte holding
-// the index bits b0a b0b b1a b1b b2a b2b of two neighbouring weights) -> (G[idx_a], G[idx_b]) as fp32,
+// Image of the decode kernel's shared-memory table, built once at pack time: entry e (a byte holding the
+// indices of two neighbouring weights as nibbles, idx_b << 4 | idx_a) -> (G[idx_a], G[idx_b]) as fp32,
 // replicated into one 8-byte slot per lane (entry stride 256 bytes).
 __global__ void build_lut_table_kernel(const PackedHeader *hdr, uint8_t *table)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= 256 * 32) return;
     const int e = i >> 5, l = i & 31;
-    const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
-    const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
+    const int ia = e & 7, ib = (e >> 4) & 7;
     *reinterpret_cast<float2 *>(table + e * 256 + l * 8) = make_float2(hdr->lut_levels[ia], hdr->lut_levels[ib]);
 }
 
@@ -230,7 +229,7 @@ __global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ld
 #pragma unroll
     for (int q = 0; q < 7; ++q) T[q] = hdr->lut_thresholds[q];
     const int zero_idx = hdr->lut_zero_idx;
-    uint32_t p0 = 0, p1 = 0, p2 = 0;
+    uint32_t wd[3] = {0u, 0u, 0u};
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         float x[16];
@@ -256,15 +255,17 @@ __global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ld
                 for (int l = 0; l < 7; ++l) idx += (y > T[l]) ? 1 : 0;
             }
             const int i = h * 16 + q;
-            p0 |= (uint32_t)(idx & 1) << lut3_bitpos(0, i);
-            p1 |= (uint32_t)((idx >> 1) & 1) << lut3_bitpos(1, i);
-            p2 |= (uint32_t)((idx >> 2) & 1) << lut3_bitpos(2, i);
+#pragma unroll
+            for (int b = 0; b < 3; ++b) {
+                int word, pos;
+                lut3_locate(b, i, word, pos);                      // all indices are compile-time constants here
+                wd[word] |= (uint32_t)((idx >> b) & 1) << pos;
+            }
         }
     }
-    // device layout: 448-byte blocks per (row, 1024-weight slice); bit order inside a word per lut3_bitpos
-    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 0, K)) = p0;
-    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 1, K)) = p1;
-    *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, 2, K)) = p2;
+    // device layout: 448-byte blocks per (row, 1024-weight slice); bit order inside the word triplet per lut3_locate
+#pragma unroll
+    for (int p = 0; p < 3; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = wd[p];
 }
 
 cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
@@ -281,21 +282,18 @@ cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, i
 
 // NVFP4 view of the LUT3 codes (Sec. 2.3): level -> nearest E2M1 value, element signs
 // flipped under a negative block scale, block scale |d|, same tensor scale.
-// One thread per plane word (32 weights).  The three plane words are merged into bytes that hold the six
-// index bits of a weight pair (as in the decode kernel); a 64-entry shared-memory table maps such a byte to
-// the byte of two E2M1 codes, in three variants: positive scale, negative scale (sign bits of non-zero codes
-// flipped), zero scale (all codes zero).  Pair q = 4g + j of the word is byte j of the word rotated by 2g,
-// and is output byte q of the row's 16 code bytes, so each merged word gives one output word.
+// One thread per word triplet (32 weights).  A selector byte holds the indices of a weight pair as nibbles;
+// a small shared-memory table maps such a byte to the byte of two E2M1 codes, in three variants: positive
+// scale, negative scale (sign bits of non-zero codes flipped), zero scale (all codes zero).  Pair q of the
+// triplet is byte q % 4 of selector word q / 4 and output byte q of the row's 16 code bytes.
 __global__ void __launch_bounds__(256) autocast_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
                                                        int64_t K, uint8_t *codes, uint8_t *sf)
 {
-    __shared__ uint8_t table[3][64];                // [variant][pair pattern] -> two E2M1 codes
+    __shared__ uint8_t table[3][128];               // [variant][idx_b << 4 | idx_a] -> two E2M1 codes
     const uint32_t amap = hdr->autocast_map;
-    if (threadIdx.x < 192) {
-        const int v = threadIdx.x >> 6, e = threadIdx.x & 63;
-        const int ia = (e & 1) | ((e >> 1) & 2) | ((e >> 2) & 4);
-        const int ib = ((e >> 1) & 1) | ((e >> 2) & 2) | ((e >> 3) & 4);
-        uint32_t ca = (amap >> (4 * ia)) & 0xFu, cb = (amap >> (4 * ib)) & 0xFu;
+    for (int i = threadIdx.x; i < 3 * 128; i += blockDim.x) {
+        const int v = i >> 7, e = i & 127;
+        uint32_t ca = (amap >> (4 * (e & 7))) & 0xFu, cb = (amap >> (4 * ((e >> 4) & 7))) & 0xFu;
         if (v == 1) { if (ca & 7u) ca ^= 8u; if (cb & 7u) cb ^= 8u; }
         if (v == 2) { ca = 0u; cb = 0u; }
         table[v][e] = (uint8_t)(ca | (cb << 4));
@@ -306,18 +304,17 @@ __global__ void __launch_bounds__(256) autocast_kernel(const PackedHeader *hdr, 
     if (i >= N * nw) return;
     const int64_t r = i / nw;
     const int j = (int)(i - r * nw);
-    const uint32_t p0 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 0, K));
-    const uint32_t p1 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 1, K));
-    const uint32_t p2 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 2, K));
+    const uint32_t w0 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 0, K));
+    const uint32_t w1 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 1, K));
+    const uint32_t w2 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 2, K));
     const uint32_t d2 = *reinterpret_cast<const unsigned short *>(lut + lut_scale_offset(r, j * 2, K));
-    uint32_t out[4];
+    uint32_t sel[4], out[4];
+    lut3_selectors(w0, w1, w2, sel);
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         const uint32_t d8 = (g < 2) ? (d2 & 0xFFu) : (d2 >> 8);            // pairs 0..7 are block 0, 8..15 block 1
         const uint8_t *tab = table[d8 == 0u ? 2 : ((d8 & 0x80u) ? 1 : 0)];
-        const uint32_t a = __funnelshift_r(p0, p0, 2 * g), b = __funnelshift_r(p1, p1, 2 * g),
-                       c = __funnelshift_r(p2, p2, 2 * g);
-        const uint32_t u = (a & 0x03030303u) | (b & 0x0C0C0C0Cu) | (c & 0x30303030u);
+        const uint32_t u = sel[g];
         out[g] = (uint32_t)tab[u & 0xFFu] | ((uint32_t)tab[(u >> 8) & 0xFFu] << 8) |
                  ((uint32_t)tab[(u >> 16) & 0xFFu] << 16) | ((uint32_t)tab[u >> 24] << 24);
     }
@@ -367,12 +364,18 @@ __global__ void export_lut3_kernel(const PackedHeader *hdr, const uint8_t *lut, 
     if (i == 0 && s_out) *s_out = hdr->s;
     if (i >= N * nw) return;
     const int64_t r = i / nw, j = i % nw;
+    uint32_t wd[3];
+#pragma unroll
+    for (int p = 0; p < 3; ++p) wd[p] = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, p, K));
 #pragma unroll
     for (int p = 0; p < 3; ++p) {
-        const uint32_t w = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, p, K));
         uint32_t c = 0;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) c |= ((w >> lut3_bitpos(p, i)) & 1u) << i;      // canonical: LSB-first
+        for (int i = 0; i < 32; ++i) {
+            int word, pos;
+            lut3_locate(p, i, word, pos);
+            c |= ((wd[word] >> pos) & 1u) << i;                                      // canonical: LSB-first bit-planes
+        }
         planes_out[(r * 3 + p) * nw + j] = c;
     }
     scales_out[r * (K / 16) + 2 * j] = lut[lut_scale_offset(r, 2 * j, K)];
@@ -421,14 +424,19 @@ __global__ void import_lut3_kernel(const uint32_t *planes_in, const uint8_t *sca
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N * nw) return;
     const int64_t r = i / nw, j = i % nw;
+    uint32_t wd[3] = {0u, 0u, 0u};
 #pragma unroll
     for (int p = 0; p < 3; ++p) {
-        const uint32_t c = planes_in[(r * 3 + p) * nw + j];                        // canonical: LSB-first
-        uint32_t w = 0;
+        const uint32_t c = planes_in[(r * 3 + p) * nw + j];                        // canonical: LSB-first bit-planes
 #pragma unroll
-        for (int b = 0; b < 32; ++b) w |= ((c >> b) & 1u) << lut3_bitpos(p, b);
-        *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = w;
+        for (int i = 0; i < 32; ++i) {
+            int word, pos;
+            lut3_locate(p, i, word, pos);
+            wd[word] |= ((c >> i) & 1u) << pos;
+        }
     }
+#pragma unroll
+    for (int p = 0; p < 3; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = wd[p];
     lut[lut_scale_offset(r, 2 * j, K)] = scales_in[r * (K / 16) + 2 * j];
     lut[lut_scale_offset(r, 2 * j + 1, K)] = scales_in[r * (K / 16) + 2 * j + 1];
 }
