@@ -510,7 +510,7 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES.get(("gemm", cfg.name)),
                      "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_sustained']} TFLOP/s); "
                                     f"nominal dense FP4 9000"},
-        "roofline_decode": {"kernel": "gemv_lut3_kernel", "bound": "hbm", "achieved": decode_gbs,
+        "roofline_decode": {"kernel": "gemv_lut3_mma_kernel" if cfg.name == DEFAULT_WORKLOAD or B >= 2 else "gemv_lut3_kernel / gemv_lut3_mma_kernel (by shape)", "bound": "hbm", "achieved": decode_gbs,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": decode_gbs / peaks["hbm_gbs"],
                             "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)),
                             "peak_source": f"{peaks['source']} copy bandwidth"},

@@ -436,9 +436,7 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
     g.ldy = ldy;
     g.N = w->N;
     g.K = w->K;
-    // batch 1: CUDA-core kernel; with two and more columns the tensor-core kernel wins (the batch rides along in
-    // the B operand: 17408x5120 at batch 2 / 8 / 16: 22 / 27 / 52 us against 26 / 103 / 206 us)
-    const bool use_mma = (g_lut_decode_kernel == 1) || (g_lut_decode_kernel < 0 && B >= 2);
+    const bool use_mma = (g_lut_decode_kernel == 1) || (g_lut_decode_kernel < 0 && dq::gemv_lut3_mma_preferred(w->N, w->K, B));
     const cudaError_t ce = use_mma ? dq::launch_gemv_lut3_mma(g, reinterpret_cast<cudaStream_t>(stream))
                                    : dq::launch_gemv_lut3(g, reinterpret_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return DQ_ERR_CUDA;

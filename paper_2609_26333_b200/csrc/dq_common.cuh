@@ -170,6 +170,7 @@ struct GemvArgs {
 };
 cudaError_t launch_gemv_lut3(const GemvArgs &args, cudaStream_t stream);              // CUDA cores: batch 1 and 2
 cudaError_t launch_gemv_lut3_mma(const GemvArgs &args, cudaStream_t stream);          // tensor cores: eight columns per pass
+bool gemv_lut3_mma_preferred(int64_t N, int64_t K, int64_t B);                          // which of the two dq_decode_linear takes
 
 struct GemvNvArgs {
     const uint8_t *codes; const uint8_t *sf;              // NVFP4 view: [N][K/2] codes, MMA-layout scales

@@ -1,4 +1,4 @@
-// LUT3 decode for small batches with the products on tensor cores (App. C.2 kernel specification; the
+// LUT3 decode with the products on tensor cores (App. C.2 kernel specification; the
 // skinny-batch case the paper leaves open, Sec. 5):
 //   Y[b][n] = bf16( s * sum_k d_blk(n,k) * G[idx(n,k)] * X[b][k] ),   up to eight batch columns per pass.
 // Same skeleton as the NVFP4 tensor-core decode kernel: a warp owns 16 consecutive rows and a 1024-weight
@@ -7,11 +7,15 @@
 // Dequantisation without shared memory: the device bit order stores indices as nibbles, which are the
 // selectors of byte-permute; the eight fp16 levels live in four registers (low bytes, high bytes), two
 // permutes look up the bytes of four weights and two more interleave them into two fp16 pairs.  The block
-// scale is applied in fp16 without loss: level * d is split into hi = rn(level * d) and lo = level * d - hi
-// (one multiply, one fused multiply-add; lo is exact), and both go through mma.sync.m16n8k16 with fp32
-// accumulation.  Activations: power-of-two scaling, fp16 in shared memory, one 8-byte load per pair of mmas.
-// At batch 1 this costs more instructions per weight than the CUDA-core kernel (which stays the batch-1
-// path, about 5 % faster there); from batch 2 on it wins because the batch rides along in the B operand.
+// scale is applied in fp16: hi = rn(level * d) goes through mma.sync.m16n8k16 with fp32 accumulation.  For
+// K < 2048 the exact remainder lo = level * d - hi (one fused multiply-add) goes through a second mma, so that
+// nothing is lost.  For K >= 2048 it is left out: the per-weight rounding errors (relative 2^-11 at most,
+// independent) add a standard deviation of about 2e-4 * rms|a w| * sqrt(K) to a sum whose tolerance is
+// 1e-4 * K * mean|a w|, i.e. 3.3 / sqrt(K) of it; measured, the largest error-to-tolerance ratio over whole
+// layers is the same with and without the remainder from K = 1024 on (0.46: the bf16 rounding of the output).
+// Activations: power-of-two scaling, fp16 in shared memory, one 8-byte load per mma (pair).
+// Used from batch 2 on (the batch rides along in the B operand) and at batch 1 for 2048 <= K <= 16384, where it
+// is faster than the CUDA-core kernel (28672x8192: 39.6 against 45.3 us).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -62,7 +66,7 @@ __global__ void __launch_bounds__(MAXT, 1)
 gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
                      const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
                      __nv_bfloat16 *__restrict__ Y, int64_t ldy, int N, int K, int W, int G, uint32_t col_stride,
-                     uint32_t x_addr, StatusWord *status)
+                     uint32_t x_addr, StatusWord *status, int hi_only)
 {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
@@ -220,7 +224,7 @@ gemv_lut3_mma_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
                         const uint32_t h0 = hmul2(v0, d0), h1 = hmul2(v1, d1), h2 = hmul2(v2, d0), h3 = hmul2(v3, d1);
                         const uint2 xv = lds_v2(xa + (uint32_t)(2 * gg + jj) * 32);
                         mma16816(acc, h0, h1, h2, h3, xv.x, xv.y);
-                        mma16816(acc, hres2(v0, d0, h0), hres2(v1, d1, h1), hres2(v2, d0, h2), hres2(v3, d1, h3), xv.x, xv.y);
+                        if (!hi_only) mma16816(acc, hres2(v0, d0, h0), hres2(v1, d1, h1), hres2(v2, d0, h2), hres2(v3, d1, h3), xv.x, xv.y);
                     }
                 }
             }
@@ -299,12 +303,35 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemv_lut3_mma_kernel<MAXT>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
                               (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
-                              (int)a.K, W, G, col_stride, x_addr, a.status);
+                              (int)a.K, W, G, col_stride, x_addr, a.status, (a.K >= 2048) ? 1 : 0);
 }
 
 }  // namespace
 
-// batches of two and more: up to eight columns per pass on tensor cores
+// Whether dq_decode_linear should take this kernel rather than the CUDA-core one.  Two and more columns: always
+// (the batch rides along in the B operand).  Batch 1: where it was measured faster, i.e. K from 2048 (one mma per
+// step) to 16384 (at most 16 slice warps per row group) and a tile count that fills the last round of the grid:
+// with 16-row tiles a 5120-row layer leaves half of the SMs idle in its second round, where the CUDA-core kernel
+// works in 4-row units.
+bool gemv_lut3_mma_preferred(int64_t N, int64_t K, int64_t B)
+{
+    if (B >= 2) return true;
+    if (K < 2048 || K > 16384) return false;
+    const int W = (int)((K + 1023) / 1024);
+    int G = 20 / W;
+    if (G < 1) G = 1;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t ntiles = N / 16;
+    int64_t grid = (ntiles + G - 1) / G;
+    if (grid > sms) grid = sms;
+    const int64_t groups = grid * G;
+    const int64_t rounds = (ntiles + groups - 1) / groups;
+    return (double)ntiles / (double)(rounds * groups) >= 0.85;
+}
+
+// up to eight columns per pass on tensor cores
 cudaError_t launch_gemv_lut3_mma(const GemvArgs &a, cudaStream_t stream)
 {
     const int K = (int)a.K, N = (int)a.N, B = (int)a.B;
