@@ -303,7 +303,7 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemv_lut3_mma_kernel<MAXT>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
                               (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
-                              (int)a.K, W, G, col_stride, x_addr, a.status, (a.K >= 2048) ? 1 : 0);
+                              (int)a.K, W, G, col_stride, x_addr, a.status, 0);
 }
 
 }  // namespace

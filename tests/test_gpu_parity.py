@@ -344,6 +344,75 @@ def test_decode_lut3_tensor_core_kernel_parity(dq, oracle, N, K, seed, B):
     check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 tensor-core decode {B}x{N}x{K}")
 
 
+def _sparse_patterns(K, seed):
+    """Activation rows on which a sum of K products is dominated by a handful of them: 1, 2, 3, 8 and 32 non-zeros
+    with random bf16 values and with +-1, two columns of one 16-block that cancel, two columns far apart."""
+    g = torch.Generator().manual_seed(seed)
+    rows = []
+    for nnz in (1, 2, 3, 8, 32):
+        for signs_only in (False, True):
+            x = torch.zeros(K)
+            pos = torch.randperm(K, generator=g)[:nnz]
+            if signs_only:
+                x[pos] = torch.randint(0, 2, (nnz,), generator=g).float() * 2 - 1
+            else:
+                x[pos] = torch.randn(nnz, generator=g) * torch.exp2(torch.randint(-3, 4, (nnz,), generator=g).float())
+            rows.append(x)
+    for blk, i, j in ((0, 0, 1), (K // 32, 3, 12), (K // 16 - 1, 15, 14)):      # +1 / -1 inside one block
+        x = torch.zeros(K)
+        x[16 * blk + i], x[16 * blk + j] = 1.0, -1.0
+        rows.append(x)
+    x = torch.zeros(K)
+    x[5], x[700] = 1.0, 1.0
+    rows.append(x)
+    x = torch.zeros(K)
+    x[K - 1], x[K // 2] = 3.0, -3.0
+    rows.append(x)
+    while len(rows) % 8:
+        rows.append(rows[len(rows) % 5])
+    return torch.stack(rows).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("N,K,seed", [(2048, 2048, 95), (1024, 4096, 96), (512, 8192, 97), (256, 5120, 98)])
+@pytest.mark.parametrize("B", [1, 2, 8])
+def test_decode_sparse_and_cancelling_activations(dq, oracle, N, K, seed, B):
+    """Per-element bound on inputs where nothing averages out: every product must be exact up to fp32
+    accumulation, so a few non-zero activations (or two that cancel) meet the same bound as dense rows."""
+    W, ref = _layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    P = _sparse_patterns(K, seed + 1)
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(P), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    Pd = P.to(DEV)
+    got = torch.cat([dq.decode_linear(w, Pd[i:i + B]) for i in range(0, P.shape[0], B)])
+    _status_ok(dq)
+    check_outputs(_f64(got), Yr, S, f"decode, sparse / cancelling activations, batch {B}, {N}x{K}")
+    # a single non-zero activation of 1.0 reads one dequantised column: exact after the bf16 rounding
+    What = oracle.dequant_lut3(ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    for k in (0, 17, K // 2 + 5, K - 1):
+        x = torch.zeros(1, K, dtype=torch.bfloat16)
+        x[0, k] = 1.0
+        y = _f64(dq.decode_linear(w, x.to(DEV)))[0]
+        want = torch.from_numpy(What[:, k]).to(torch.bfloat16).float().numpy().astype(np.float64)
+        assert np.array_equal(y, want), f"one-hot column {k}"
+
+
+def test_decode_lut3_wide_range_activations(dq, oracle):
+    """Activations spanning many binades (the kernel rescales them by a power of two into fp16), strided and
+    guarded outputs."""
+    N, K = 400, 2048
+    W, ref = _layer(oracle, N, K, 90)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    for B in (1, 5):
+        g = torch.Generator().manual_seed(91 + B)
+        X = (torch.randn(B, K, generator=g) * torch.exp2(torch.randint(-20, 12, (B, K), generator=g).float())).to(torch.bfloat16)
+        Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+        out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+        dq.decode_linear(w, X.to(DEV), out=out[:, :N])
+        _status_ok(dq)
+        assert torch.all(out[:, N:] == -3.0)
+        check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 decode, wide-range activations, batch {B}")
+
+
 def test_decode_one_hot_and_strided(dq, oracle):
     N, K = 256, 512
     W, ref = _layer(oracle, N, K, 64)
