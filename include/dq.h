@@ -15,9 +15,12 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream); work is
  *     enqueued on it and the call returns without synchronising;
  *   - nothing is allocated on the device; scratch comes from the caller;
- *   - shapes: K % 128 == 0, N % 16 == 0 (else DQ_ERR_SHAPE); row strides in
+ *   - shapes: K % 128 == 0, N % 16 == 0, and K <= 32768 for a handle that holds a
+ *     LUT encoding (else DQ_ERR_SHAPE); row strides in
  *     elements, multiples of 8; device pointers 16-byte aligned, `packed_dev`
  *     and `workspace_dev` 1024-byte aligned (else DQ_ERR_ALIGN);
+ *   - a handle belongs to the device that was current when it was packed; calls that
+ *     use it with another device current return DQ_ERR_INVALID_ARG;
  *   - NaN/Inf in tensors give unspecified values, never a fault;
  *   - the device must be compute capability 10.0 (else DQ_ERR_ARCH).
  */
@@ -49,7 +52,8 @@ enum dq_status {
 enum dq_format {
     DQ_FMT_NVFP4 = 1,            /* NVFP4 round-to-nearest of the master weights   */
     DQ_FMT_LUT3 = 2,             /* LUT3 round-to-nearest of the master weights    */
-    DQ_FMT_NVFP4_FROM_LUT3 = 4   /* NVFP4 view re-quantised from the LUT3 codes    */
+    DQ_FMT_NVFP4_FROM_LUT3 = 4,  /* NVFP4 view re-quantised from the LUT3 codes    */
+    DQ_FMT_LUT2 = 8              /* LUT2 round-to-nearest of the master weights    */
 };
 
 enum dq_dtype { DQ_DT_BF16 = 0, DQ_DT_FP32 = 1 };
@@ -60,10 +64,9 @@ const char *dq_status_string(int status);
 
 /*
  * Size of the device buffer dq_pack_weights needs for the requested encodings.
- * Storage follows App. A.3 "Storage cost": NVFP4 4.5 bit and LUT3 3.5 bit per
- * weight (codes plus one FP8 scale per 16 weights), plus a 1 KiB header, a 64 KiB
- * lookup table for the decode kernel (LUT3 only), padding of the NVFP4 scale tiles to
- * 256 rows and of LUT3 rows to a multiple of 1024 weights.
+ * Storage follows App. A.3 "Storage cost": NVFP4 4.5 bit, LUT3 3.5 bit and LUT2 2.5 bit
+ * per weight (codes plus one FP8 scale per 16 weights), plus a 1 KiB header, padding of
+ * the NVFP4 scale tiles to 256 rows and of LUT rows to a multiple of 1024 weights.
  * `formats` must contain at most one of DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3;
  * DQ_FMT_NVFP4_FROM_LUT3 implies DQ_FMT_LUT3.
  */
@@ -77,7 +80,9 @@ int dq_packed_bytes(int64_t N, int64_t K, unsigned formats, size_t *bytes_host);
  *   block scale   d_b = E4M3(extreme_b / (6 s)) per 16 weights along K; for LUT3
  *                 it carries the sign of the block's maximum-magnitude weight;
  *   NVFP4 code    nearest E2M1 value of w / (s d_b);
- *   LUT3 index    nearest level of the 8-entry fp16 codebook, stored bit-planed.
+ *   LUT3 index    nearest level of the 8-entry fp16 codebook, stored bit-planed;
+ *   LUT2 index    nearest level of the paper's 4-level LUT2A16 grid {-3.6517, 0, 2.5227, 6}
+ *                 rounded to fp16, same signed block scale rule.
  *   DQ_FMT_NVFP4_FROM_LUT3 derives the NVFP4 codes from the LUT3 indices
  *   (Sec. 2.3 autocast) instead of from W.
  * W_dev: device, row-major, row stride ldw elements, dtype per `w_dtype`.
@@ -161,11 +166,26 @@ int dq_prefill_linear_static(const dq_weights *w, const void *A_dev, int64_t M, 
  * Decode linear (Sec. 1.1 "memory-bound decode", App. C.2 "Kernel specification"):
  *   Y[b][n] = bf16( sum_k X[b][k] * W~[n][k] ),  W~ = s * d_b * codebook[idx],
  * a weight-only mat-vec / skinny GEMM on the handle's LUT3 weights with raw bf16
- * activations and fp32 accumulation.  1 <= B <= 64.
+ * activations.  1 <= B <= 64.
+ * Arithmetic: the products codebook[idx] * x are formed exactly (fp16 levels and the
+ * activations, scaled by one power of two into fp16, on tensor cores) and summed in fp32 per
+ * 16-weight block; the block sum is multiplied by d_b and accumulated in fp32; s is applied to
+ * the total.  Nothing is rounded before the fp32 accumulation, so the error per output is a few
+ * fp32 rounding errors of sum_k |x w| plus the bf16 rounding of the result, for any activation
+ * pattern.  An activation more than 2^28 times smaller in magnitude than the largest activation
+ * of the same call (of the same group of four rows of X) loses low bits or reads as zero.
  * X_dev: B x K bf16, row stride ldx; Y_dev: B x N bf16, row stride ldy.
  */
 int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
                      void *Y_dev, int64_t ldy, void *stream);
+
+/*
+ * The same decode on the handle's LUT2 weights (App. A.3 "LUT formats": 4 levels, 2.5 bit per
+ * weight; App. C.2; Table 1's LUT2 rows).  Needs DQ_FMT_LUT2 in the handle.  Arguments, arithmetic
+ * and limits as dq_decode_linear.
+ */
+int dq_decode_linear_lut2(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
+                          void *Y_dev, int64_t ldy, void *stream);
 
 /*
  * The same decode on the handle's NVFP4 view (weight-only NVFP4A16, Sec. 2.3 and Table 1
@@ -213,8 +233,8 @@ int dq_decode_linear_host(const dq_weights *w, const void *X_host, int64_t B, in
  *     codes  uint8[N][K/2]  element 2j in the low nibble, 2j+1 in the high nibble,
  *            code = sign<<3 | index into {0,.5,1,1.5,2,3,4,6} (App. A.3 "NVFP4")
  *     scales uint8[N][K/16] E4M3
- *   DQ_FMT_LUT3:
- *     codes  uint32[N][3][K/32] bit-planes (App. C.2): bit i (LSB = 0) of word j of
+ *   DQ_FMT_LUT3 (b = 3) / DQ_FMT_LUT2 (b = 2):
+ *     codes  uint32[N][b][K/32] bit-planes (App. C.2): bit i (LSB = 0) of word j of
  *            plane p is bit p of the index of weight 32*j + i
  *     scales uint8[N][K/16] signed E4M3, zero stored as 0x00
  *   global_scale_dev: one float, the tensor scale s.
@@ -229,6 +249,7 @@ int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, v
  * need lut3_planes_dev / lut3_scales_dev (unused pointers may be NULL); global_scale is the tensor
  * scale s (finite, > 0), shared by both encodings.  packed_dev / packed_bytes / ownership as in
  * dq_pack_weights.  No value check is made on the codes: every bit pattern decodes to something.
+ * DQ_FMT_LUT2 cannot be imported (DQ_ERR_INVALID_ARG): it is packed from master weights only.
  */
 int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp4_codes_dev,
                         const void *nvfp4_scales_dev, const void *lut3_planes_dev,
@@ -255,6 +276,26 @@ int dq_get_status(void *stream, int *status_host, int *detail_host);
 
 /* Shape queries on a handle. */
 int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsigned *formats_host);
+
+/* ---- test hooks (the paper has no counterpart; not for production callers) ---- */
+
+/*
+ * A decode call with its launch parameters forced, so that tests reach every work split and the
+ * bounded-wait exit of the kernels without touching global state.
+ *   format  DQ_FMT_LUT3 / DQ_FMT_LUT2: the LUT decode kernel with `warps_per_group` warps sharing an
+ *           8-row tile, `groups_per_cta` such groups per CTA, `ring_stages` bulk-copy stages per
+ *           warp (each 0 = the launcher's choice; their product must fit 32 warps, stages 2..8) and
+ *           a device-side wait budget of `wait_cycles` SM clocks (0 = the default of about two
+ *           seconds).  variant 1 additionally leaves out one bulk copy (the first atom of warp 0 of
+ *           CTA 0), so that the wait for it runs out after `wait_cycles`: the kernel returns normally,
+ *           writes partial output and records DQ_ERR_TIMEOUT for dq_get_status.
+ *   format  DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3: the NVFP4A16 decode; variant 0 = the tensor-core
+ *           kernel dq_decode_linear_nvfp4 runs, 1 = the CUDA-core kernel kept for comparison.
+ * Other arguments as dq_decode_linear.
+ */
+int dq_test_decode_linear(const dq_weights *w, unsigned format, int variant, int warps_per_group,
+                          int groups_per_cta, int ring_stages, long long wait_cycles, const void *X_dev,
+                          int64_t B, int64_t ldx, void *Y_dev, int64_t ldy, void *stream);
 
 #ifdef __cplusplus
 }

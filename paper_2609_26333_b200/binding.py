@@ -13,6 +13,7 @@ _LIB_PATH = _PKG / "libdq.so"
 FMT_NVFP4 = 1
 FMT_LUT3 = 2
 FMT_NVFP4_FROM_LUT3 = 4
+FMT_LUT2 = 8
 DT_BF16 = 0
 DT_FP32 = 1
 
@@ -20,7 +21,7 @@ DT_FP32 = 1
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
-           "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_export_canonical", "dq_import_canonical",
+           "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
            "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
@@ -74,6 +75,11 @@ def lib() -> C.CDLL:
         L.dq_decode_linear_host.argtypes = [vp, vp, i64, i64, vp, i64, vp, C.c_size_t, vp]
         L.dq_decode_linear_nvfp4.restype = C.c_int
         L.dq_decode_linear_nvfp4.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_decode_linear_lut2.restype = C.c_int
+        L.dq_decode_linear_lut2.argtypes = [vp, vp, i64, i64, vp, i64, vp]
+        L.dq_test_decode_linear.restype = C.c_int
+        L.dq_test_decode_linear.argtypes = [vp, C.c_uint, C.c_int, C.c_int, C.c_int, C.c_int, C.c_longlong, vp, i64, i64,
+                                            vp, i64, vp]
         L.dq_import_canonical.restype = C.c_int
         L.dq_import_canonical.argtypes = [C.c_int64, C.c_int64, C.c_uint, vp, vp, vp, vp, C.c_float,
                                           C.POINTER(C.c_uint16), vp, C.c_size_t, vp, C.POINTER(vp)]
@@ -263,6 +269,34 @@ def decode_linear_nvfp4(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None,
     return out
 
 
+def decode_linear_lut2(w: DQWeights, X: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """dq_decode_linear_lut2: Y = X @ LUT2(W)^T, bf16 out, batch 1..64."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    B = X.shape[0]
+    if out is None:
+        out = torch.empty(B, w.N, dtype=torch.bfloat16, device=X.device)
+    _check(lib().dq_decode_linear_lut2(w.handle, X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
+                                       _stream_ptr(stream)), "dq_decode_linear_lut2")
+    return out
+
+
+def test_decode_linear(w: DQWeights, fmt: int, X: torch.Tensor, out: torch.Tensor = None, variant: int = 0,
+                       warps_per_group: int = 0, groups_per_cta: int = 0, ring_stages: int = 0, wait_cycles: int = 0,
+                       stream=None) -> torch.Tensor:
+    """dq_test_decode_linear: a decode call with forced launch parameters (test hook)."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    B = X.shape[0]
+    if out is None:
+        out = torch.empty(B, w.N, dtype=torch.bfloat16, device=X.device)
+    _check(lib().dq_test_decode_linear(w.handle, fmt, variant, warps_per_group, groups_per_cta, ring_stages,
+                                       int(wait_cycles), X.data_ptr(), B, X.stride(0), out.data_ptr(), out.stride(0),
+                                       _stream_ptr(stream)), "dq_test_decode_linear")
+    return out
+
+
+test_decode_linear.__test__ = False      # not a pytest test
+
+
 def prefill_host_staging_bytes(w: DQWeights, M: int) -> int:
     out = C.c_size_t(0)
     _check(lib().dq_prefill_host_staging_bytes(w.handle, M, C.byref(out)), "dq_prefill_host_staging_bytes")
@@ -296,7 +330,7 @@ def export_canonical(w: DQWeights, fmt: int, stream=None):
     if fmt in (FMT_NVFP4, FMT_NVFP4_FROM_LUT3):
         codes = torch.empty(w.N, w.K // 2, dtype=torch.uint8, device=dev)
     else:
-        codes = torch.empty(w.N, 3, w.K // 32, dtype=torch.int32, device=dev)
+        codes = torch.empty(w.N, 3 if fmt == FMT_LUT3 else 2, w.K // 32, dtype=torch.int32, device=dev)
     scales = torch.empty(w.N, w.K // 16, dtype=torch.uint8, device=dev)
     s = torch.empty(1, dtype=torch.float32, device=dev)
     _check(lib().dq_export_canonical(w.handle, fmt, codes.data_ptr(), scales.data_ptr(), s.data_ptr(),

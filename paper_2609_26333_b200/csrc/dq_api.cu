@@ -36,23 +36,33 @@ int check_arch()
     return DQ_OK;
 }
 
-int check_shape(int64_t N, int64_t K)
+int check_shape(int64_t N, int64_t K, unsigned formats)
 {
     if (N <= 0 || K <= 0) return DQ_ERR_SHAPE;
     if (K % 128 != 0 || N % 16 != 0) return DQ_ERR_SHAPE;
     if (N > (1ll << 30) || K > (1ll << 30)) return DQ_ERR_SHAPE;
+    // the LUT decode kernel keeps a whole activation row in shared memory
+    if ((formats & (DQ_FMT_LUT3 | DQ_FMT_LUT2 | DQ_FMT_NVFP4_FROM_LUT3)) && K > dq::kLutMaxK) return DQ_ERR_SHAPE;
     return DQ_OK;
 }
 
 int check_formats(unsigned formats)
 {
-    const unsigned all = DQ_FMT_NVFP4 | DQ_FMT_LUT3 | DQ_FMT_NVFP4_FROM_LUT3;
+    const unsigned all = DQ_FMT_NVFP4 | DQ_FMT_LUT3 | DQ_FMT_NVFP4_FROM_LUT3 | DQ_FMT_LUT2;
     if (formats == 0 || (formats & ~all)) return DQ_ERR_INVALID_ARG;
     if ((formats & DQ_FMT_NVFP4) && (formats & DQ_FMT_NVFP4_FROM_LUT3)) return DQ_ERR_INVALID_ARG;
     return DQ_OK;
 }
 
 bool valid_handle(const dq_weights *w) { return w != nullptr && w->magic == kMagic; }
+
+// the handle's buffers live on the device it was packed on; a call made with another device current
+// would hand that device's kernels foreign pointers
+bool on_handle_device(const dq_weights *w)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == w->device;
+}
 
 // Prefill workspace: NVFP4 activations (codes, MMA-layout scales); for a handle that stores only
 // LUT3 the NVFP4 view of the weights (codes, MMA-layout scales) follows, rebuilt on every call.
@@ -112,7 +122,7 @@ const char *dq_status_string(int status)
     switch (status) {
         case DQ_OK: return "ok";
         case DQ_ERR_INVALID_ARG: return "invalid argument";
-        case DQ_ERR_SHAPE: return "unsupported shape (need K % 128 == 0, N % 16 == 0)";
+        case DQ_ERR_SHAPE: return "unsupported shape (need K % 128 == 0, N % 16 == 0; K <= 32768 for LUT formats)";
         case DQ_ERR_ALIGN: return "misaligned pointer or stride";
         case DQ_ERR_WORKSPACE: return "buffer too small";
         case DQ_ERR_ARCH: return "device is not compute capability 10.0";
@@ -128,7 +138,7 @@ int dq_packed_bytes(int64_t N, int64_t K, unsigned formats, size_t *bytes_host)
     if (!bytes_host) return DQ_ERR_INVALID_ARG;
     int st = check_formats(formats);
     if (st != DQ_OK) return st;
-    st = check_shape(N, K);
+    st = check_shape(N, K, formats);
     if (st != DQ_OK) return st;
     *bytes_host = dq::packed_layout(N, K, formats).total;
     return DQ_OK;
@@ -142,7 +152,7 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
     if (w_dtype != DQ_DT_BF16 && w_dtype != DQ_DT_FP32) return DQ_ERR_INVALID_ARG;
     int st = check_formats(formats);
     if (st != DQ_OK) return st;
-    st = check_shape(N, K);
+    st = check_shape(N, K, formats);
     if (st != DQ_OK) return st;
     if (ldw < K || ldw % 8 != 0) return DQ_ERR_ALIGN;
     if (!aligned(W_dev, 16) || !aligned(packed_dev, 1024)) return DQ_ERR_ALIGN;
@@ -171,12 +181,18 @@ int dq_pack_weights(const void *W_dev, int w_dtype, int64_t N, int64_t K, int64_
             return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_LUT3) {
-        if (L.lut_bytes != (size_t)N * K / 16 * 7) {       // partial last slice: padding must read as zero
+        if (K % dq::kLutSlice != 0) {       // partial last slice: padding must read as zero
             if (cudaMemsetAsync(base + L.lut_off, 0, L.lut_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
         }
-        if (dq::launch_pack_lut3(W_dev, w_dtype, N, K, ldw, hdr, base + L.lut_off, s) != cudaSuccess)
+        if (dq::launch_pack_lut(3, W_dev, w_dtype, N, K, ldw, hdr, base + L.lut_off, s) != cudaSuccess)
             return DQ_ERR_CUDA;
-        if (dq::launch_build_lut_table(hdr, base + L.lut_table_off, s) != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    if (formats & DQ_FMT_LUT2) {
+        if (K % dq::kLutSlice != 0) {
+            if (cudaMemsetAsync(base + L.lut2_off, 0, L.lut2_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+        }
+        if (dq::launch_pack_lut(2, W_dev, w_dtype, N, K, ldw, hdr, base + L.lut2_off, s) != cudaSuccess)
+            return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
         if (dq::launch_autocast(hdr, base + L.lut_off, N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
@@ -207,9 +223,10 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
     if (!packed_dev || !out_host) return DQ_ERR_INVALID_ARG;
     int st = check_formats(formats);
     if (st != DQ_OK) return st;
-    st = check_shape(N, K);
+    st = check_shape(N, K, formats);
     if (st != DQ_OK) return st;
     if (!(global_scale > 0.0f) || !std::isfinite(global_scale)) return DQ_ERR_INVALID_ARG;
+    if (formats & DQ_FMT_LUT2) return DQ_ERR_INVALID_ARG;          // LUT2 is packed from master weights only
     if (formats & DQ_FMT_NVFP4_FROM_LUT3) formats |= DQ_FMT_LUT3;
     if ((formats & DQ_FMT_NVFP4) && (!nvfp4_codes_dev || !nvfp4_scales_dev)) return DQ_ERR_INVALID_ARG;
     if ((formats & DQ_FMT_LUT3) && (!lut3_planes_dev || !lut3_scales_dev)) return DQ_ERR_INVALID_ARG;
@@ -239,13 +256,12 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
             return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_LUT3) {
-        if (L.lut_bytes != (size_t)N * K / 16 * 7 && cudaMemsetAsync(base + L.lut_off, 0, L.lut_bytes, s) != cudaSuccess)
+        if (K % dq::kLutSlice != 0 && cudaMemsetAsync(base + L.lut_off, 0, L.lut_bytes, s) != cudaSuccess)
             return DQ_ERR_CUDA;
-        if (dq::launch_import_lut3(reinterpret_cast<const uint32_t *>(lut3_planes_dev),
-                                   reinterpret_cast<const uint8_t *>(lut3_scales_dev), N, K, base + L.lut_off, s) !=
+        if (dq::launch_import_lut(3, reinterpret_cast<const uint32_t *>(lut3_planes_dev),
+                                  reinterpret_cast<const uint8_t *>(lut3_scales_dev), N, K, base + L.lut_off, s) !=
             cudaSuccess)
             return DQ_ERR_CUDA;
-        if (dq::launch_build_lut_table(hdr, base + L.lut_table_off, s) != cudaSuccess) return DQ_ERR_CUDA;
     }
     if (formats & DQ_FMT_NVFP4_FROM_LUT3) {
         if (dq::launch_autocast(hdr, base + L.lut_off, N, K, base + L.nv_codes_off, base + L.nv_sf_off, s) !=
@@ -296,6 +312,7 @@ static int prefill_checks(const dq_weights *w, int64_t M, float act_global_scale
                           size_t workspace_bytes)
 {
     if (!valid_handle(w) || !workspace_dev) return DQ_ERR_INVALID_ARG;
+    if (!on_handle_device(w)) return DQ_ERR_INVALID_ARG;
     if (!has_nvfp4_view(w) && !(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
     if (M < 1 || M > (1ll << 24)) return DQ_ERR_INVALID_ARG;
     if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
@@ -332,9 +349,6 @@ int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64
     return DQ_OK;
 }
 
-static int g_gemm_probe = 0;
-int dq_debug_gemm_probe(int mode) { int old = g_gemm_probe; g_gemm_probe = mode; return old; }
-
 int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
                     const void *workspace_dev, size_t workspace_bytes, void *stream)
 {
@@ -361,7 +375,6 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
     g.N = w->N;
     g.K = w->K;
     g.status = sw;
-    g.probe = g_gemm_probe;
     if (dq::launch_gemm_nvfp4(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
@@ -379,16 +392,11 @@ int dq_prefill_linear(const dq_weights *w, const void *A_dev, int64_t M, int64_t
     return dq_prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream);
 }
 
-static int g_lut_decode_kernel = -1;    // -1 = by batch size, 0 = CUDA-core kernel, 1 = tensor-core kernel
-int dq_debug_lut3_decode_kernel(int which) { int old = g_lut_decode_kernel; g_lut_decode_kernel = which; return old; }
-static int g_nv_decode_kernel = 1;      // 1 = tensor-core kernel, 0 = CUDA-core kernel (kept for comparison)
-int dq_debug_nvfp4_decode_kernel(int which) { int old = g_nv_decode_kernel; g_nv_decode_kernel = which; return old; }
-
-int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
-                           void *stream)
+static int decode_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                        void *stream, bool tensor_cores)
 {
     if (!valid_handle(w) || !X_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
-    if (!has_nvfp4_view(w)) return DQ_ERR_INVALID_ARG;
+    if (!has_nvfp4_view(w) || !on_handle_device(w)) return DQ_ERR_INVALID_ARG;
     if (B < 1 || B > 64) return DQ_ERR_INVALID_ARG;
     if (ldx < w->K || ldy < w->N || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
     if (!aligned(X_dev, 16) || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
@@ -407,25 +415,32 @@ int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, in
     g.ldy = ldy;
     g.N = w->N;
     g.K = w->K;
-    const cudaError_t ce = g_nv_decode_kernel ? dq::launch_gemv_nvfp4_mma(g, reinterpret_cast<cudaStream_t>(stream))
-                                              : dq::launch_gemv_nvfp4(g, reinterpret_cast<cudaStream_t>(stream));
+    const cudaError_t ce = tensor_cores ? dq::launch_gemv_nvfp4_mma(g, reinterpret_cast<cudaStream_t>(stream))
+                                        : dq::launch_gemv_nvfp4(g, reinterpret_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
 
-int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
-                     void *stream)
+int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                           void *stream)
+{
+    return decode_nvfp4(w, X_dev, B, ldx, Y_dev, ldy, stream, true);
+}
+
+static int decode_lut(const dq_weights *w, unsigned format, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev,
+                      int64_t ldy, void *stream, int P, int G, int S, long long wait_cycles, int drop_first_copy = 0)
 {
     if (!valid_handle(w) || !X_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
-    if (!(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
+    if (format != DQ_FMT_LUT3 && format != DQ_FMT_LUT2) return DQ_ERR_INVALID_ARG;
+    if (!(w->formats & format) || !on_handle_device(w)) return DQ_ERR_INVALID_ARG;
     if (B < 1 || B > 64) return DQ_ERR_INVALID_ARG;
     if (ldx < w->K || ldy < w->N || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_ALIGN;
     if (!aligned(X_dev, 16) || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
     int st = check_arch();
     if (st != DQ_OK) return st;
     dq::GemvArgs g;
-    g.lut = w->base + w->layout.lut_off;
-    g.table = w->base + w->layout.lut_table_off;
+    g.bits = (format == DQ_FMT_LUT3) ? 3 : 2;
+    g.lut = w->base + (format == DQ_FMT_LUT3 ? w->layout.lut_off : w->layout.lut2_off);
     g.status = status_word_ptr();
     if (!g.status) return DQ_ERR_CUDA;
     g.hdr = reinterpret_cast<const dq::PackedHeader *>(w->base);
@@ -436,11 +451,39 @@ int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t 
     g.ldy = ldy;
     g.N = w->N;
     g.K = w->K;
-    const bool use_mma = (g_lut_decode_kernel == 1) || (g_lut_decode_kernel < 0 && dq::gemv_lut3_mma_preferred(w->N, w->K, B));
-    const cudaError_t ce = use_mma ? dq::launch_gemv_lut3_mma(g, reinterpret_cast<cudaStream_t>(stream))
-                                   : dq::launch_gemv_lut3(g, reinterpret_cast<cudaStream_t>(stream));
+    g.force_P = P;
+    g.force_G = G;
+    g.force_S = S;
+    g.wait_cycles = wait_cycles;
+    g.drop_first_copy = drop_first_copy;
+    const cudaError_t ce = dq::launch_gemv_lut(g, reinterpret_cast<cudaStream_t>(stream));
+    if (ce == cudaErrorInvalidValue) return DQ_ERR_INVALID_ARG;
     if (ce != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                     void *stream)
+{
+    return decode_lut(w, DQ_FMT_LUT3, X_dev, B, ldx, Y_dev, ldy, stream, 0, 0, 0, 0);
+}
+
+int dq_decode_linear_lut2(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev, int64_t ldy,
+                          void *stream)
+{
+    return decode_lut(w, DQ_FMT_LUT2, X_dev, B, ldx, Y_dev, ldy, stream, 0, 0, 0, 0);
+}
+
+int dq_test_decode_linear(const dq_weights *w, unsigned format, int variant, int warps_per_group, int groups_per_cta,
+                          int ring_stages, long long wait_cycles, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev,
+                          int64_t ldy, void *stream)
+{
+    if (format == DQ_FMT_NVFP4 || format == DQ_FMT_NVFP4_FROM_LUT3)
+        return decode_nvfp4(w, X_dev, B, ldx, Y_dev, ldy, stream, variant == 0);
+    if (warps_per_group < 0 || groups_per_cta < 0 || ring_stages < 0 || ring_stages > 8 || wait_cycles < 0)
+        return DQ_ERR_INVALID_ARG;
+    return decode_lut(w, format, X_dev, B, ldx, Y_dev, ldy, stream, warps_per_group, groups_per_cta, ring_stages,
+                      wait_cycles, variant == 1 ? 1 : 0);
 }
 
 int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, void *scales_dev,
@@ -457,11 +500,12 @@ int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, v
             return DQ_ERR_CUDA;
         return DQ_OK;
     }
-    if (format == DQ_FMT_LUT3) {
-        if (!(w->formats & DQ_FMT_LUT3)) return DQ_ERR_INVALID_ARG;
-        if (dq::launch_export_lut3(hdr, w->base + w->layout.lut_off, w->N, w->K,
-                                   reinterpret_cast<uint32_t *>(codes_dev), reinterpret_cast<uint8_t *>(scales_dev),
-                                   global_scale_dev, s) != cudaSuccess)
+    if (format == DQ_FMT_LUT3 || format == DQ_FMT_LUT2) {
+        if (!(w->formats & format)) return DQ_ERR_INVALID_ARG;
+        const bool l3 = (format == DQ_FMT_LUT3);
+        if (dq::launch_export_lut(l3 ? 3 : 2, hdr, w->base + (l3 ? w->layout.lut_off : w->layout.lut2_off), w->N, w->K,
+                                  reinterpret_cast<uint32_t *>(codes_dev), reinterpret_cast<uint8_t *>(scales_dev),
+                                  global_scale_dev, s) != cudaSuccess)
             return DQ_ERR_CUDA;
         return DQ_OK;
     }

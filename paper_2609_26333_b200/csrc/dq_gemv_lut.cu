@@ -1,0 +1,590 @@
+// LUT3 / LUT2 weight-only decode (App. C.2 "Kernel specification"; the skinny-batch case the paper leaves open, Sec. 5):
+//   Y[b][n] = bf16( s * sum_blk d_blk(n) * sum_{k in blk} G[idx(n,k)] * X[b][k] ),   up to four batch columns per pass.
+//
+// Arithmetic.  Every product G[idx] * x is exact: the fp16 codebook levels go to the tensor cores unscaled
+// (mma.sync.m16n8k16, fp32 accumulation), the bf16 activations are scaled by one power of two into fp16 (no
+// rounding for any element within 2^28 of the largest of the pass), and one mma contracts exactly one 16-weight
+// block per row, so that the signed E4M3 block scale multiplies the block's fp32 sum afterwards, in fp32:
+//   acc += d_blk * (sum of 16 exact products).
+// Nothing is rounded before the fp32 accumulation, whatever the activations look like (dense, sparse, cancelling).
+//
+// Work split.  A row tile is 8 rows.  The 16 rows of the mma's A operand are the 8 rows of the tile against two
+// neighbouring blocks b, b+1; the B operand holds block b of the activations in columns 0-3 (one per batch column)
+// and block b+1 in columns 4-7, so accumulator entries (row g, column c) and (row g+8, column 4+c) are the two
+// halves of one output and the cross terms are dropped.  Lane (g, t) supplies weights 4t .. 4t+3 of both blocks of
+// row g, which is how the device layout stores them (dq_common.cuh).  A group of P warps shares a tile, warp w
+// taking 1024-weight slices w, w+P, .. (P = 1: a warp owns whole tiles and stores its outputs itself; otherwise
+// the last warp of the group to arrive adds the partial tiles in a fixed order); G groups per CTA, one or two
+// CTAs per SM, tiles dealt round robin.
+//
+// Memory.  Every warp streams its own chunks (8 rows x 1024 weights = two atoms, 3584 B for LUT3) through a ring of
+// S bulk copies (cp.async.bulk + mbarrier) in shared memory, refilling a stage as soon as its words sit in registers.
+// Dequantisation is register-only: the stored words are byte-permute selectors after one AND, two permutes fetch the
+// low and high bytes of four levels from the codebook held in four registers and two more interleave them into two
+// fp16 pairs.  The 256 block scales of an atom are converted to fp32 once per warp (eight per lane) and parked in a
+// small per-warp buffer; a lane reads its row's scales and its B fragments with 16-byte loads, two mmas per load.
+//
+// What bounds it.  On this GPU a warp instruction of the integer / logic / permute class occupies the issue port of
+// its SM sub-partition for two cycles (measured: 8 PRMT + 8 FFMA take 24 cycles, not 16), so the kernel is bound by
+// instruction issue: about 8 permutes, 2 logic ops, 2 shifts, 1 mma, 4 FFMA and 2 shared loads per 8 weights of a lane.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "dq_common.cuh"
+#include "dq_tcgen05.cuh"
+
+namespace dq {
+
+namespace {
+
+constexpr int kSlots = 4;                         // cross-warp reduction slots per row group
+constexpr uint32_t kSmemLimit = 227 * 1024;
+constexpr uint32_t kSmemLimitHalf = 113 * 1024;   // two CTAs per SM
+constexpr int kMaxWarps = 24;
+constexpr int kMaxGroups = 12;
+constexpr uint32_t kScaleBufBytes = 1152;         // per warp: 8 rows x 36 floats (32 block scales + 4 of padding)
+
+// shared-memory map (byte offsets from the start of dynamic shared memory) and work split, filled in by the launcher
+struct LutPlan {
+    int P, G, S;                      // warps per row group, row groups per CTA, ring stages per warp
+    uint32_t bar_off;                 // ring barriers: [warp][S] x 8 B
+    uint32_t red_off;                 // reduction slots: [G][kSlots][P][32] floats
+    uint32_t sbuf_off;                // per warp: 8 rows x 32 fp32 block scales of the atom being worked on
+    uint32_t ring_off;                // [warp][S][atom]
+    uint32_t x_off;                   // [cols][col_stride] fp16 activations
+    uint32_t col_stride;
+    long long wait_cycles;
+    int drop_first_copy;              // test hook: CTA 0 / warp 0 never requests its first atom, so that its wait runs out
+};
+
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// 8-byte shared-memory load at base + OFF (the offset is an immediate of the instruction)
+template <int OFF>
+__device__ __forceinline__ uint2 lds_v2_at(uint32_t base)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(base), "n"(OFF));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint4 lds_v4_at(uint32_t base)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base), "n"(OFF) : "memory");
+    return v;
+}
+// four signed E4M3 bytes -> four floats (exact)
+__device__ __forceinline__ float4 e4m3x4_to_f32(uint32_t four)
+{
+    uint32_t h01, h23;
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, lo;\n\tcvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+        : "=r"(h01), "=r"(h23) : "r"(four));
+    float4 r;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(r.x), "=f"(r.y) : "r"(h01));
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(r.z), "=f"(r.w) : "r"(h23));
+    return r;
+}
+__device__ __forceinline__ void sts_v4f(uint32_t addr, float4 v)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ float4 lds_v4f_at(uint32_t base)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+%5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(base), "n"(OFF));
+    return v;
+}
+
+// bounded mbarrier wait with back-off between polls
+__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long budget)
+{
+    if (tc::mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (true) {
+        __nanosleep(20);
+        if (tc::mbar_try(bar, parity)) return true;
+        if ((++it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > budget) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+// byte permute, selector taken as it is (nibbles with the top bit clear select bytes 0-7 of {a, b})
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+
+struct Codebook { uint32_t tl0, tl1, th0, th1; };    // low bytes of levels 0-3 / 4-7, high bytes of levels 0-3 / 4-7
+
+// Two neighbouring blocks of the atom (selector word `sel`: low half the first block, high half the second) against
+// their activations xv: one mma, then the two block scales d0, d1 (fp32) on the two block sums.
+__device__ __forceinline__ void block_pair(uint32_t sel, uint32_t x0, uint32_t x1, float d0, float d1, const Codebook &cb,
+                                           float (&acc)[4])
+{
+    const uint32_t u1 = sel >> 16;
+    const uint32_t lo0 = prmt(cb.tl0, cb.tl1, sel), hi0 = prmt(cb.th0, cb.th1, sel);
+    const uint32_t a0 = prmt(lo0, hi0, 0x5140u), a2 = prmt(lo0, hi0, 0x7362u);     // row g, first block
+    const uint32_t lo1 = prmt(cb.tl0, cb.tl1, u1), hi1 = prmt(cb.th0, cb.th1, u1);
+    const uint32_t a1 = prmt(lo1, hi1, 0x5140u), a3 = prmt(lo1, hi1, 0x7362u);     // "row g+8": second block
+    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    mma16816(c, a0, a1, a2, a3, x0, x1);
+    acc[0] = fmaf(c[0], d0, acc[0]);
+    acc[1] = fmaf(c[1], d0, acc[1]);
+    acc[2] = fmaf(c[2], d1, acc[2]);
+    acc[3] = fmaf(c[3], d1, acc[3]);
+}
+
+// One word group (32 weights of this lane: four of each of the blocks 8 WI .. 8 WI + 7 of the atom).  The group's
+// activations (this lane's column, block parity and quarter of a block) are 32 contiguous bytes at xa + 256 WI, its eight
+// block scales eight contiguous floats at sa + 32 WI: 16-byte loads serve two mmas each.
+template <int BITS, int WI>
+__device__ __forceinline__ void group_dot(const uint32_t (&w)[BITS], uint32_t xa, uint32_t sa, const Codebook &cb,
+                                          float (&acc)[4])
+{
+    uint32_t sel[4];
+    lut_selectors<BITS>(w, sel);
+    const uint4 xA = lds_v4_at<WI * 256>(xa), xB = lds_v4_at<WI * 256 + 16>(xa);
+    const float4 dA = lds_v4f_at<WI * 32>(sa), dB = lds_v4f_at<WI * 32 + 16>(sa);
+    block_pair(sel[0], xA.x, xA.y, dA.x, dA.y, cb, acc);
+    block_pair(sel[1], xA.z, xA.w, dA.z, dA.w, cb, acc);
+    block_pair(sel[2], xB.x, xB.y, dB.x, dB.y, cb, acc);
+    block_pair(sel[3], xB.z, xB.w, dB.z, dB.w, cb, acc);
+}
+
+// One atom of this lane's row: BITS index words x 4 word groups, against the fp16 activations at shared address xa
+// (this lane's column and block parity; layout in the kernel) and the row's 32 block scales as fp32 at shared address sa.
+template <int BITS>
+__device__ __forceinline__ void atom_dot(const uint4 (&pw)[BITS], uint32_t xa, uint32_t sa, const Codebook &cb,
+                                         float (&acc)[4])
+{
+    uint32_t w[BITS];
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) w[p] = pw[p].x;
+    group_dot<BITS, 0>(w, xa, sa, cb, acc);
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) w[p] = pw[p].y;
+    group_dot<BITS, 1>(w, xa, sa, cb, acc);
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) w[p] = pw[p].z;
+    group_dot<BITS, 2>(w, xa, sa, cb, acc);
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) w[p] = pw[p].w;
+    group_dot<BITS, 3>(w, xa, sa, cb, acc);
+}
+
+// Activations of one column in shared memory, fp16.  An atom (512 weights, 32 blocks) takes 1024 bytes ordered
+// [word group 4][block parity 2][quarter t 4][block pair 4][4 weights], so that the four B fragments lane (., t) needs for
+// the four mmas of a word group (blocks 8 wi + 2a + parity, weights 4t .. 4t+3, a = 0..3) are 32 contiguous bytes.
+// Byte offset of the eight weights 8 i .. 8 i + 7 (a quarter pair t = 2h, 2h+1 of one block; the second quarter 32 bytes on):
+__device__ __forceinline__ uint32_t x_offset(int i)
+{
+    const uint32_t atom = (uint32_t)i >> 6, bb = ((uint32_t)i >> 1) & 31u, h = (uint32_t)i & 1u;
+    return atom * 1024u + (bb >> 3) * 256u + (bb & 1u) * 128u + h * 64u + ((bb >> 1) & 3u) * 8u;
+}
+
+__device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
+
+template <int BITS, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
+gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
+                const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
+                __nv_bfloat16 *__restrict__ Y, int64_t ldy, int N, int K, LutPlan L, StatusWord *status)
+{
+    constexpr uint32_t kAtom = (uint32_t)lut_atom_bytes(BITS);
+    constexpr uint32_t kChunk = 2u * kAtom;                 // one ring stage: 8 rows x 1024 weights
+    constexpr uint32_t kPlanes = (uint32_t)lut_plane_bytes(BITS);
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw);
+    int *sync_words = reinterpret_cast<int *>(smem_raw + 64);                           // [G][kSlots] x (generation, count)
+    float *xmax_s = reinterpret_cast<float *>(smem_raw + 512);                          // 32 per-warp maxima
+    float *red = reinterpret_cast<float *>(smem_raw + L.red_off);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
+    const int P = L.P, G = L.G, S = L.S;
+    const int grp = warp / P;
+    const int w = warp - grp * P;
+    const int g = lane >> 2, t = lane & 3;
+    const int nslices = (int)lut_slices(K);
+    const int kpad = nslices * kLutSlice;
+
+    // ---- this warp's ring: S stages of one chunk each, one barrier per stage; nobody else touches them
+    const uint32_t ring0 = win0 + L.ring_off + (uint32_t)warp * (uint32_t)S * kChunk;
+    const uint32_t bars0 = win0 + L.bar_off + (uint32_t)warp * (uint32_t)S * 8u;
+    if (lane == 0) {
+        for (int i = 0; i < S; ++i) tc::mbar_init(bars0 + 8u * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x < kMaxGroups * kSlots * 2) sync_words[threadIdx.x] = 0;
+    if (threadIdx.x == 0) *abort_flag = 0;
+    __syncwarp();
+
+    // slices w, w + P, .. of every tile this warp's group owns
+    const int ns = (w < nslices) ? (nslices - w + P - 1) / P : 0;
+    const int ntiles = N / kLutAtomRows;
+    const int stride = gridDim.x * G;
+    const int first = blockIdx.x * G + grp;
+    const size_t slice_step = (size_t)P * 4u * kAtom;         // bytes between slices s and s + P of one tile
+    auto tile_base = [&](int tile) {                           // chunk (tile, slice w)
+        return lut + (((size_t)(tile >> 1) * nslices + w) * 4u + (size_t)(tile & 1) * 2u) * kAtom;
+    };
+    // producer state (lane 0): next chunk to request
+    const uint8_t *psrc = tile_base(first);
+    int pslice = 0, ptile = (ns > 0) ? first : ntiles, pstage = 0;       // ptile >= ntiles: nothing left to request
+    auto advance = [&]() {
+        if (++pslice == ns) { pslice = 0; ptile += stride; psrc = tile_base(ptile); }
+        else psrc += slice_step;
+        if (++pstage == S) pstage = 0;
+    };
+    auto issue_next = [&]() {
+        tc::mbar_expect_tx(bars0 + 8u * pstage, kChunk);
+        tc::bulk_load(ring0 + (uint32_t)pstage * kChunk, psrc, kChunk, bars0 + 8u * pstage);
+        advance();
+    };
+    // The weights are constant data: start streaming before waiting for the kernel ahead of this one.
+    if (lane == 0) {
+        const bool drop = L.drop_first_copy && blockIdx.x == 0 && warp == 0;
+        for (int i = 0; i < S && ptile < ntiles; ++i) {
+            if (drop && i == 0) advance();                      // test hook: this chunk is never requested
+            else issue_next();
+        }
+    }
+    const uint4 cbv = *reinterpret_cast<const uint4 *>(BITS == 3 ? hdr->lut_prmt : hdr->lut2_prmt);
+    const Codebook cb = {cbv.x, cbv.y, cbv.z, cbv.w};
+    const float s_w = hdr->s;
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ---- activations of this pass: one read from global memory (raw bf16 parked in shared memory, largest
+    //      magnitude on the way), then power-of-two scale -> fp16 in place
+    uint8_t *xh = smem_raw + L.x_off;
+    float m = 0.0f;
+    for (int c = 0; c < cols; ++c) {
+        const uint4 *xp = reinterpret_cast<const uint4 *>(X + (int64_t)(b0 + c) * ldx);
+        for (int i = threadIdx.x; i < kpad / 8; i += blockDim.x) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);                 // the padding of a short last slice reads as zero
+            if (i < K / 8) v = __ldg(xp + i);
+            // |bf16| pairs compare like unsigned integers once the sign bits are cleared
+            const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+            const uint32_t hi = max(max(a0 >> 16, a1 >> 16), max(a2 >> 16, a3 >> 16));
+            const uint32_t lo = max(max(a0 & 0xFFFFu, a1 & 0xFFFFu), max(a2 & 0xFFFFu, a3 & 0xFFFFu));
+            m = fmaxf(m, __uint_as_float(max(hi, lo) << 16));
+            uint8_t *dst = xh + (size_t)c * L.col_stride + x_offset(i);
+            *reinterpret_cast<uint2 *>(dst) = make_uint2(v.x, v.y);
+            *reinterpret_cast<uint2 *>(dst + 32) = make_uint2(v.z, v.w);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) xmax_s[warp] = m;
+    __syncthreads();
+    m = (lane < nwarps) ? xmax_s[lane] : 0.0f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    int ex = (int)((__float_as_uint(m) >> 23) & 0xFFu) - 127;           // floor(log2(max)); -127 for zero / subnormal
+    ex = max(-100, min(100, ex));
+    const float xscale = __uint_as_float((uint32_t)(127 + 14 - ex) << 23);   // 2^(14 - ex)
+    const float xinv = __uint_as_float((uint32_t)(127 - 14 + ex) << 23);
+    for (int c = 0; c < cols; ++c) {
+        for (int i = threadIdx.x; i < kpad / 8; i += blockDim.x) {        // every thread converts what it parked itself
+            uint8_t *px = xh + (size_t)c * L.col_stride + x_offset(i);
+            const uint2 va = *reinterpret_cast<const uint2 *>(px), vb = *reinterpret_cast<const uint2 *>(px + 32);
+            const uint32_t ww[4] = {va.x, va.y, vb.x, vb.y};
+            uint32_t r[4];
+#pragma unroll
+            for (int z = 0; z < 4; ++z) {
+                const __half2 h = __floats2half2_rn(__uint_as_float(ww[z] << 16) * xscale,
+                                                    __uint_as_float(ww[z] & 0xFFFF0000u) * xscale);
+                r[z] = *reinterpret_cast<const uint32_t *>(&h);
+            }
+            *reinterpret_cast<uint2 *>(px) = make_uint2(r[0], r[1]);
+            *reinterpret_cast<uint2 *>(px + 32) = make_uint2(r[2], r[3]);
+        }
+    }
+    __syncthreads();
+    const float out_scale = s_w * xinv;
+    // B operand of this lane: column g % 4 (column 0 where the pass has fewer), block parity g / 4, weights 4t .. 4t+3
+    const int colsel = ((g & 3) < cols) ? (g & 3) : 0;
+    const uint32_t xlane = win0 + L.x_off + (uint32_t)colsel * L.col_stride + (uint32_t)(g >> 2) * 128u + (uint32_t)t * 32u +
+                           (uint32_t)w * (kLutSlice * 2u);
+    const uint32_t lane_plane = (uint32_t)lane * 16u;
+    // this warp's fp32 scale buffer: 8 rows x 32 blocks; lane l converts bytes 8 l .. 8 l + 7 of the atom's scale bytes
+    // (row l / 4, blocks 8 (l % 4) ..), which land at float 8 l of the buffer: row-major like the bytes
+    const uint32_t sbuf = win0 + L.sbuf_off + (uint32_t)warp * kScaleBufBytes;
+    const uint32_t srow = sbuf + (uint32_t)g * 144u;                        // rows 36 floats apart: conflict-free reads
+    const uint32_t swr = sbuf + (uint32_t)(lane >> 2) * 144u + (uint32_t)(lane & 3) * 32u;
+    const uint32_t sync0 = win0 + 64u + (uint32_t)grp * kSlots * 8u;
+
+    bool ok = true;
+    int stage = 0;
+    uint32_t phase = 0;
+    int tile = first;
+    for (int it = 0; tile < ntiles; ++it, tile += stride) {
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        uint32_t xa = xlane;
+        for (int sl = 0; sl < ns; ++sl, xa += (uint32_t)P * (kLutSlice * 2u)) {
+            // one lane polls (with back-off) so that waiting warps do not flood the shared-memory pipe; after a wait
+            // that ran out every warp keeps walking the same iterations without touching data
+            if (ok) {
+                uint32_t good = 1;
+                if (lane == 0) good = ring_wait(bars0 + 8u * stage, phase, abort_flag, L.wait_cycles) ? 1u : 0u;
+                ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+            }
+            if (ok) {
+                const uint32_t base = ring0 + (uint32_t)stage * kChunk;
+                uint4 pw[BITS];
+                uint2 s8;
+                // atom 0: index words to registers; the warp converts the atom's 256 block scales to fp32 once (8 per
+                // lane) and parks them in its scale buffer, from which every lane reads its row's
+                pw[0] = lds_v4_at<0>(base + lane_plane);
+                pw[1] = lds_v4_at<512>(base + lane_plane);
+                if (BITS == 3) pw[BITS - 1] = lds_v4_at<1024>(base + lane_plane);
+                s8 = lds_v2_at<(int)kPlanes>(base + (uint32_t)lane * 8u);
+                __syncwarp();                                          // everybody is done with the buffer's last contents
+                sts_v4f(swr, e4m3x4_to_f32(s8.x));
+                sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
+                __syncwarp();
+                atom_dot<BITS>(pw, xa, srow, cb, acc);
+                pw[0] = lds_v4_at<(int)kAtom>(base + lane_plane);
+                pw[1] = lds_v4_at<(int)kAtom + 512>(base + lane_plane);
+                if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(base + lane_plane);
+                s8 = lds_v2_at<(int)(kAtom + kPlanes)>(base + (uint32_t)lane * 8u);
+                // the stage is in registers: refill it with the chunk S steps ahead
+                __syncwarp();
+                if (lane == 0 && ptile < ntiles) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    issue_next();
+                }
+                sts_v4f(swr, e4m3x4_to_f32(s8.x));
+                sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
+                __syncwarp();
+                atom_dot<BITS>(pw, xa + kLutAtomK * 2u, srow, cb, acc);
+            }
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        // halves of an output: (row g, column c) in lanes t < 2 and (row g + 8, column 4 + c) in lanes t >= 2
+        const float v0 = acc[0] + __shfl_xor_sync(0xffffffffu, acc[2], 2);
+        const float v1 = acc[1] + __shfl_xor_sync(0xffffffffu, acc[3], 2);
+        if (P == 1) {
+            // the warp owns the whole tile: lanes t < 2 hold (row g, columns 2t, 2t+1)
+            if (ok && t < 2) {
+                const int row = tile * kLutAtomRows + g;
+                if (2 * t < cols) Y[(int64_t)(b0 + 2 * t) * ldy + row] = __float2bfloat16_rn(v0 * out_scale);
+                if (2 * t + 1 < cols) Y[(int64_t)(b0 + 2 * t + 1) * ldy + row] = __float2bfloat16_rn(v1 * out_scale);
+            }
+            continue;
+        }
+        // ---- cross-warp sum: last-arriving warp of the group adds the P partial tiles in order and stores
+        const int slot = it & (kSlots - 1);
+        const uint32_t gen_addr = sync0 + (uint32_t)slot * 8u;
+        int *cnt = sync_words + (grp * kSlots + slot) * 2 + 1;
+        if (ok) {
+            uint32_t good = 1;
+            if (lane == 0) {
+                const uint32_t want = (uint32_t)(it / kSlots);
+                long long t0 = 0;
+                uint32_t spins = 0;
+                while (lds_u32_volatile(gen_addr) != want) {
+                    if ((++spins & 255u) == 0u) {
+                        if (t0 == 0) t0 = clock64();
+                        if (*abort_flag || clock64() - t0 > L.wait_cycles) { *abort_flag = 1; good = 0; break; }
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+        }
+        float *rbuf = red + (size_t)((grp * kSlots + slot) * P) * 32;
+        if (t < 2) *reinterpret_cast<float2 *>(rbuf + w * 32 + g * 4 + 2 * t) = make_float2(v0, v1);
+        __syncwarp();
+        int prev = 0;
+        if (lane == 0) { fence_cta(); prev = atomicAdd(cnt, 1); }
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev == P - 1) {
+            fence_cta();
+            float tot = 0.0f;
+            for (int ww = 0; ww < P; ++ww) tot += *reinterpret_cast<const volatile float *>(rbuf + ww * 32 + lane);
+            const int col = lane & 3, row = tile * kLutAtomRows + (lane >> 2);
+            if (ok && col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot * out_scale);
+            __syncwarp();
+            if (lane == 0) {
+                *cnt = 0;
+                fence_cta();
+                asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(gen_addr), "r"((uint32_t)(it / kSlots + 1)) : "memory");
+            }
+        }
+    }
+    if (*abort_flag) {
+        // a wait ran out: let copies in flight land before the CTA's shared memory is handed on, then report
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        if (lane == 0) {
+            atomicExch(&status->status, (int)DQ_ERR_TIMEOUT);
+            atomicExch(&status->detail, 0x36000 | (int)blockIdx.x);
+        }
+    }
+}
+
+template <int BITS, int MAXT, int MINB>
+cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int threads, const LutPlan &L, uint32_t smem,
+                       cudaStream_t stream)
+{
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_lut_kernel<BITS, MAXT, MINB>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
+                              (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
+                              (int)a.K, L, a.status);
+}
+
+}  // namespace
+
+// Shared-memory map for P x G warps with S ring stages and `cols` activation columns; returns the bytes needed.
+static uint32_t plan_smem(int bits, int K, int P, int G, int S, int cols, LutPlan &L)
+{
+    const int nwarps = P * G;
+    const uint32_t chunk = 2u * (uint32_t)lut_atom_bytes(bits);
+    L.P = P; L.G = G; L.S = S;
+    L.bar_off = 1024;
+    L.red_off = 2048;
+    const uint32_t red_bytes = (uint32_t)nwarps * kSlots * 32 * 4;
+    L.sbuf_off = (L.red_off + red_bytes + 127u) & ~127u;
+    L.ring_off = L.sbuf_off + (uint32_t)nwarps * kScaleBufBytes;
+    L.x_off = (L.ring_off + (uint32_t)nwarps * S * chunk + 127u) & ~127u;
+    L.col_stride = (uint32_t)lut_slices(K) * kLutSlice * 2u + 16u;    // padded K in fp16; 16 mod 32 keeps two columns' 16-byte loads on different banks
+    return L.x_off + (uint32_t)cols * L.col_stride;
+}
+
+struct Split { int P, G, ctas, S, cols; };
+
+// Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA, one
+// or two CTAs per SM.  Two smaller CTAs are preferred: with half of an SM's registers and shared memory each, the
+// CTAs of the next launch in the stream (programmatic dependent launch) move in while this launch drains, and their
+// set-up and first copies overlap its tail.  Modelled time of a launch: the larger of what the busiest SM has to issue
+// (tiles x (chunks per tile + a charge per warp for the cross-warp sum, none when a warp owns whole tiles)) and what one
+// warp has to get through on its own; all `want_cols` columns in one pass where shared memory allows.  The constants
+// come from sweeps over (P, G) on 17408x5120, 8192x5120, 5120x17408 and 28672x8192.
+static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols)
+{
+    const int nslices = (int)lut_slices(K);
+    const int64_t ntiles = N / kLutAtomRows;
+    double best = 1e300;
+    Split sp = {1, 1, 1, 2, 1};
+    LutPlan tmp;
+    for (int ctas = 2; ctas >= 1; --ctas) {
+        const int max_warps = ctas == 2 ? 12 : kMaxWarps;
+        const uint32_t smem_cap = ctas == 2 ? kSmemLimitHalf : kSmemLimit;
+        for (int p = 1; p <= nslices && p <= max_warps; ++p) {
+            const int ns_max = (nslices + p - 1) / p;                               // slices of warp 0
+            for (int gg = 1; gg <= kMaxGroups && gg * p <= max_warps; ++gg) {
+                int cols = want_cols;
+                while (cols > 1 && plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > smem_cap) --cols;
+                if (plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > smem_cap) continue;
+                const int S = plan_smem(bits, (int)K, p, gg, 3, cols, tmp) <= smem_cap ? 3 : 2;
+                // CTAs actually launched, CTAs and tiles on the busiest SM, rounds of the busiest group
+                const int64_t need = (ntiles + gg - 1) / gg;
+                const int64_t grid = need < (int64_t)sms * ctas ? need : (int64_t)sms * ctas;
+                const int64_t rounds = (ntiles + grid * gg - 1) / (grid * gg);
+                const double rounds_eff = 0.5 * ((double)rounds + (double)ntiles / (double)(grid * gg));   // SMs finish unevenly, not in lockstep
+                const int64_t ctas_on_sm = (grid + sms - 1) / sms;
+                const double warps = (double)(ctas_on_sm * gg * p);
+                const double per_tile = (double)ns_max * p + (p > 1 ? 0.25 * p : 0.0);       // chunks (slowest warp x P) + cross-warp sum
+                const double sm_work = (double)(ctas_on_sm * gg) * rounds_eff * per_tile / (warps < 16.0 ? warps / 16.0 : 1.0);
+                const double alone = rounds_eff * 8.0 * ns_max;                              // one warp's own chain
+                const int passes = (want_cols + cols - 1) / cols;
+                // ties: two CTAs per SM, then more warps; a second pass over the weights costs a whole launch
+                const double cost = (double)passes * (sm_work > alone ? sm_work : alone) - 1e-3 * ctas * gg * p - (ctas == 2 ? 0.05 : 0.0);
+                if (cost < best) { best = cost; sp = {p, gg, ctas, S, cols}; }
+            }
+        }
+    }
+    return sp;
+}
+
+template <int BITS>
+static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, int threads, int ctas, const LutPlan &L,
+                               uint32_t smem, cudaStream_t stream)
+{
+    if (ctas == 2 && threads <= 384) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    if (threads <= 768) return launch_one<BITS, 768, 1>(a, b0, cols, grid, threads, L, smem, stream);
+    return launch_one<BITS, 1024, 1>(a, b0, cols, grid, threads, L, smem, stream);
+}
+
+// up to four columns per pass
+cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
+{
+    const int K = (int)a.K, N = (int)a.N, B = (int)a.B;
+    if (a.bits != 2 && a.bits != 3) return cudaErrorInvalidValue;
+    if (K > kLutMaxK) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int want_cols = B < 4 ? B : 4;
+    Split sp = choose_split(a.bits, N, K, sms, want_cols);
+    LutPlan L;
+    if (a.force_P > 0 && a.force_G > 0) {
+        if (a.force_P * a.force_G > 32 || a.force_G > kMaxGroups) return cudaErrorInvalidValue;
+        sp.P = a.force_P; sp.G = a.force_G;
+        sp.S = a.force_S > 0 ? a.force_S : 2;
+        sp.cols = want_cols;
+        sp.ctas = (sp.P * sp.G <= 12 && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) <= kSmemLimitHalf) ? 2 : 1;
+        while (sp.cols > 1 && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) > kSmemLimit) --sp.cols;
+    } else if (a.force_S > 0) {
+        sp.S = a.force_S;
+    }
+    const uint32_t smem_cap = sp.ctas == 2 ? kSmemLimitHalf : kSmemLimit;
+    if (plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) > smem_cap) return cudaErrorInvalidValue;
+    const int threads = sp.P * sp.G * 32;
+    const int64_t need = ((int64_t)N / kLutAtomRows + sp.G - 1) / sp.G;
+    const int grid = (int)(need < (int64_t)sms * sp.ctas ? need : (int64_t)sms * sp.ctas);
+    L.wait_cycles = a.wait_cycles > 0 ? a.wait_cycles : tc::kWaitBudgetCycles;
+    L.drop_first_copy = a.drop_first_copy;
+    for (int b0 = 0; b0 < B; b0 += sp.cols) {
+        const int cols = (B - b0 < sp.cols) ? (B - b0) : sp.cols;
+        const uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
+        const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.ctas, L, smem, stream)
+                                            : launch_bits<2>(a, b0, cols, grid, threads, sp.ctas, L, smem, stream);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace dq

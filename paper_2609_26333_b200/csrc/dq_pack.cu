@@ -107,6 +107,26 @@ __global__ void pack_header_kernel(PackedHeader *hdr, Codebook8 cb)
     hdr->lut_thresholds[7] = __int_as_float(0x7f800000);
     hdr->lut_zero_idx = zero_idx;
     hdr->autocast_map = amap;
+    // LUT2A16 grid (App. A.3 "LUT formats"), rounded to fp16
+    const float grid2[4] = {-3.6517f, 0.0f, 2.5227f, 6.0f};
+    for (int j = 0; j < 4; ++j) {
+        const __half h = __float2half_rn(grid2[j]);
+        hdr->lut2_f16[j] = __half_as_ushort(h);
+        hdr->lut2_levels[j] = __half2float(h);
+        if (hdr->lut2_levels[j] == 0.0f) hdr->lut2_zero_idx = j;
+    }
+    for (int j = 0; j < 3; ++j)
+        hdr->lut2_thresholds[j] = __fmul_rn(__fadd_rn(hdr->lut2_levels[j], hdr->lut2_levels[j + 1]), 0.5f);
+    hdr->lut2_thresholds[3] = __int_as_float(0x7f800000);
+    for (int q = 0; q < 4; ++q) { hdr->lut_prmt[q] = 0u; hdr->lut2_prmt[q] = 0u; }
+    for (int j = 0; j < 8; ++j) {
+        hdr->lut_prmt[j >> 2] |= (hdr->lut_f16[j] & 0xFFu) << (8 * (j & 3));
+        hdr->lut_prmt[2 + (j >> 2)] |= ((hdr->lut_f16[j] >> 8) & 0xFFu) << (8 * (j & 3));
+    }
+    for (int j = 0; j < 4; ++j) {
+        hdr->lut2_prmt[0] |= (hdr->lut2_f16[j] & 0xFFu) << (8 * j);
+        hdr->lut2_prmt[2] |= ((hdr->lut2_f16[j] >> 8) & 0xFFu) << (8 * j);
+    }
 }
 
 cudaError_t launch_pack_header(PackedHeader *hdr, const uint16_t *codebook_f16_host, cudaStream_t stream)
@@ -193,88 +213,98 @@ cudaError_t launch_pack_nvfp4(const void *W, int w_dtype, int64_t N, int64_t K, 
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------- decode pair table
+// ---------------------------------------------------------------- LUT pack
 
-// Image of the decode kernel's shared-memory table, built once at pack time: entry e (a byte holding the
-// indices of two neighbouring weights as nibbles, idx_b << 4 | idx_a) -> (G[idx_a], G[idx_b]) as fp32,
-// replicated into one 8-byte slot per lane (entry stride 256 bytes).
-__global__ void build_lut_table_kernel(const PackedHeader *hdr, uint8_t *table)
-{
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= 256 * 32) return;
-    const int e = i >> 5, l = i & 31;
-    const int ia = e & 7, ib = (e >> 4) & 7;
-    *reinterpret_cast<float2 *>(table + e * 256 + l * 8) = make_float2(hdr->lut_levels[ia], hdr->lut_levels[ib]);
-}
-
-cudaError_t launch_build_lut_table(const PackedHeader *hdr, uint8_t *table_dev, cudaStream_t stream)
-{
-    build_lut_table_kernel<<<32, 256, 0, stream>>>(hdr, table_dev);
-    return cudaGetLastError();
-}
-
-// --------------------------------------------------------------- LUT3 pack
-
-// One thread quantises 32 consecutive weights (two 16-blocks) and emits one word of each bit-plane.
 template <bool FP32IN>
-__global__ void pack_lut3_kernel(const void *W, int64_t N, int64_t K, int64_t ldw, const PackedHeader *hdr,
-                                 uint8_t *lut)
+__device__ __forceinline__ void load4(const void *base, int64_t row, int64_t k0, int64_t ld, float (&x)[4])
 {
-    const int64_t nw = K / 32;
+    if (FP32IN) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(base) + row * ld + k0));
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else {
+        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(base) + row * ld + k0));
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    }
+}
+
+// the larger magnitude of two signed values; equal magnitudes: the positive one
+__device__ __forceinline__ float signed_extreme(float m, float v)
+{
+    return (fabsf(v) > fabsf(m) || (fabsf(v) == fabsf(m) && v > m)) ? v : m;
+}
+
+// LUT3 / LUT2 round-to-nearest (App. A.3 "LUT formats").  Four neighbouring threads (t = 0..3) quantise the 128
+// weights 128 q .. 128 q + 127 of one row: thread t holds weights 4t .. 4t+3 of each of the eight 16-blocks, which is
+// exactly what its word group of the device layout stores; the block extreme is found across the four threads.
+template <bool FP32IN, int BITS>
+__global__ void __launch_bounds__(128) pack_lut_kernel(const void *W, int64_t N, int64_t K, int64_t ldw,
+                                                       const PackedHeader *hdr, uint8_t *lut)
+{
+    const int64_t nq = K / 128;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N * nw) return;
-    const int64_t r = i / nw, j = i % nw;
+    const int64_t quad = i >> 2;
+    const int t = (int)(i & 3);
+    const bool live = quad < N * nq;                      // whole quads are live or not; shuffles stay inside a quad
+    const int64_t r = live ? quad / nq : 0, q = live ? quad % nq : 0;
     const float s = hdr->s, rc6 = hdr->rc6;
-    float T[7];
+    constexpr int NT = (1 << BITS) - 1;
+    float T[NT];
 #pragma unroll
-    for (int q = 0; q < 7; ++q) T[q] = hdr->lut_thresholds[q];
-    const int zero_idx = hdr->lut_zero_idx;
-    uint32_t wd[3] = {0u, 0u, 0u};
+    for (int l = 0; l < NT; ++l) T[l] = (BITS == 3) ? hdr->lut_thresholds[l] : hdr->lut2_thresholds[l];
+    const int zero_idx = (BITS == 3) ? hdr->lut_zero_idx : hdr->lut2_zero_idx;
+    uint32_t wd[BITS];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        float x[16];
-        load16<FP32IN>(W, r, j * 32 + h * 16, ldw, x);
+    for (int p = 0; p < BITS; ++p) wd[p] = 0u;
+    uint32_t sc_lo = 0u, sc_hi = 0u;
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+        float x[4];
+        load4<FP32IN>(W, r, q * 128 + bb * 16 + t * 4, ldw, x);
         // the block's maximum-magnitude weight with its sign; equal magnitudes: the positive one
-        float m = x[0];
-#pragma unroll
-        for (int q = 1; q < 16; ++q) {
-            const float v = x[q];
-            if (fabsf(v) > fabsf(m) || (fabsf(v) == fabsf(m) && v > m)) m = v;
-        }
+        float m = signed_extreme(signed_extreme(x[0], x[1]), signed_extreme(x[2], x[3]));
+        m = signed_extreme(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = signed_extreme(m, __shfl_xor_sync(0xffffffffu, m, 2));
         uint32_t d8 = f32_to_e4m3(__fmul_rn(m, rc6));
         if ((d8 & 0x7Fu) == 0u) d8 = 0u;
-        lut[lut_scale_offset(r, j * 2 + h, K)] = (uint8_t)d8;
+        if (bb < 4) sc_lo |= d8 << (8 * bb); else sc_hi |= d8 << (8 * (bb - 4));
         const float rr = (d8 != 0u) ? __frcp_rn(__fmul_rn(s, e4m3_to_f32(d8))) : 0.0f;
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
+        for (int n4 = 0; n4 < 4; ++n4) {
             int idx = zero_idx;
             if (d8 != 0u) {
-                const float y = __fmul_rn(x[q], rr);
+                const float y = __fmul_rn(x[n4], rr);
                 idx = 0;
 #pragma unroll
-                for (int l = 0; l < 7; ++l) idx += (y > T[l]) ? 1 : 0;
+                for (int l = 0; l < NT; ++l) idx += (y > T[l]) ? 1 : 0;
             }
-            const int i = h * 16 + q;
 #pragma unroll
-            for (int b = 0; b < 3; ++b) {
+            for (int b = 0; b < BITS; ++b) {
                 int word, pos;
-                lut3_locate(b, i, word, pos);                      // all indices are compile-time constants here
+                lut_locate<BITS>(bb, n4, b, word, pos);            // compile-time constants after unrolling
                 wd[word] |= (uint32_t)((idx >> b) & 1) << pos;
             }
         }
     }
-    // device layout: 448-byte blocks per (row, 1024-weight slice); bit order inside the word triplet per lut3_locate
+    if (!live) return;
 #pragma unroll
-    for (int p = 0; p < 3; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = wd[p];
+    for (int p = 0; p < BITS; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, q, t, p, K, BITS)) = wd[p];
+    if (t == 0) *reinterpret_cast<uint2 *>(lut + lut_scale_offset(r, q * 8, K, BITS)) = make_uint2(sc_lo, sc_hi);
 }
 
-cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
-                             const PackedHeader *hdr, uint8_t *lut_dev, cudaStream_t stream)
+cudaError_t launch_pack_lut(int bits, const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw,
+                            const PackedHeader *hdr, uint8_t *lut_dev, cudaStream_t stream)
 {
-    const int64_t total = N * (K / 32);
+    const int64_t total = N * (K / 128) * 4;
     const unsigned blocks = (unsigned)((total + 127) / 128);
-    if (w_dtype == DQ_DT_FP32) pack_lut3_kernel<true><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
-    else pack_lut3_kernel<false><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+    const bool f32 = (w_dtype == DQ_DT_FP32);
+    if (bits == 3) {
+        if (f32) pack_lut_kernel<true, 3><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+        else pack_lut_kernel<false, 3><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+    } else {
+        if (f32) pack_lut_kernel<true, 2><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+        else pack_lut_kernel<false, 2><<<blocks, 128, 0, stream>>>(W, N, K, ldw, hdr, lut_dev);
+    }
     return cudaGetLastError();
 }
 
@@ -282,10 +312,11 @@ cudaError_t launch_pack_lut3(const void *W, int w_dtype, int64_t N, int64_t K, i
 
 // NVFP4 view of the LUT3 codes (Sec. 2.3): level -> nearest E2M1 value, element signs
 // flipped under a negative block scale, block scale |d|, same tensor scale.
-// One thread per word triplet (32 weights).  A selector byte holds the indices of a weight pair as nibbles;
-// a small shared-memory table maps such a byte to the byte of two E2M1 codes, in three variants: positive
-// scale, negative scale (sign bits of non-zero codes flipped), zero scale (all codes zero).  Pair q of the
-// triplet is byte q % 4 of selector word q / 4 and output byte q of the row's 16 code bytes.
+// One thread per word group (32 weights: four of each of eight blocks).  A selector byte holds the indices of a
+// weight pair as nibbles; a small shared-memory table maps such a byte to the byte of two E2M1 codes, in three
+// variants: positive scale, negative scale (sign bits of non-zero codes flipped), zero scale (all codes zero).
+// Selector word a holds blocks 2a (low half) and 2a+1 (high half); the thread's four codes of a block are two
+// consecutive bytes of the row's code bytes.
 __global__ void __launch_bounds__(256) autocast_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
                                                        int64_t K, uint8_t *codes, uint8_t *sf)
 {
@@ -299,34 +330,32 @@ __global__ void __launch_bounds__(256) autocast_kernel(const PackedHeader *hdr, 
         table[v][e] = (uint8_t)(ca | (cb << 4));
     }
     __syncthreads();
-    const int nw = (int)(K / 32);
+    const int64_t nq = K / 128;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N * nw) return;
-    const int64_t r = i / nw;
-    const int j = (int)(i - r * nw);
-    const uint32_t w0 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 0, K));
-    const uint32_t w1 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 1, K));
-    const uint32_t w2 = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, 2, K));
-    const uint32_t d2 = *reinterpret_cast<const unsigned short *>(lut + lut_scale_offset(r, j * 2, K));
-    uint32_t sel[4], out[4];
-    lut3_selectors(w0, w1, w2, sel);
+    const int64_t quad = i >> 2;
+    const int t = (int)(i & 3);
+    if (quad >= N * nq) return;
+    const int64_t r = quad / nq, q = quad % nq;
+    uint32_t w[3], sel[4];
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint32_t d8 = (g < 2) ? (d2 & 0xFFu) : (d2 >> 8);            // pairs 0..7 are block 0, 8..15 block 1
+    for (int p = 0; p < 3; ++p) w[p] = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, q, t, p, K, 3));
+    lut_selectors<3>(w, sel);
+    const uint2 d8x8 = *reinterpret_cast<const uint2 *>(lut + lut_scale_offset(r, q * 8, K, 3));
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+        const uint32_t d8 = ((bb < 4 ? d8x8.x : d8x8.y) >> (8 * (bb & 3))) & 0xFFu;
         const uint8_t *tab = table[d8 == 0u ? 2 : ((d8 & 0x80u) ? 1 : 0)];
-        const uint32_t u = sel[g];
-        out[g] = (uint32_t)tab[u & 0xFFu] | ((uint32_t)tab[(u >> 8) & 0xFFu] << 8) |
-                 ((uint32_t)tab[(u >> 16) & 0xFFu] << 16) | ((uint32_t)tab[u >> 24] << 24);
+        const uint32_t u = (sel[bb >> 1] >> (16 * (bb & 1))) & 0xFFFFu;
+        const unsigned short two = (unsigned short)((uint32_t)tab[u & 0xFFu] | ((uint32_t)tab[u >> 8] << 8));
+        *reinterpret_cast<unsigned short *>(codes + r * (K / 2) + q * 64 + bb * 8 + t * 2) = two;
+        if (t == (bb & 3)) sf[sf_swizzled_offset(r, q * 8 + bb, K)] = (uint8_t)(d8 & 0x7Fu);
     }
-    *reinterpret_cast<uint4 *>(codes + r * (K / 2) + (int64_t)j * 16) = make_uint4(out[0], out[1], out[2], out[3]);
-    sf[sf_swizzled_offset(r, j * 2, K)] = (uint8_t)(d2 & 0x7Fu);
-    sf[sf_swizzled_offset(r, j * 2 + 1, K)] = (uint8_t)((d2 >> 8) & 0x7Fu);
 }
 
 cudaError_t launch_autocast(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
                             int64_t K, uint8_t *codes, uint8_t *sf_swizzled, cudaStream_t stream)
 {
-    const int64_t total = N * (K / 32);
+    const int64_t total = N * (K / 128) * 4;
     autocast_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, lut_dev, N, K, codes, sf_swizzled);
     return cudaGetLastError();
 }
@@ -356,39 +385,54 @@ cudaError_t launch_export_nvfp4(const PackedHeader *hdr, const uint8_t *codes, c
     return cudaGetLastError();
 }
 
-__global__ void export_lut3_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
-                                   int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out)
+// index of weight k of row r, read from the device layout
+template <int BITS>
+__device__ __forceinline__ int lut_read_index(const uint8_t *lut, int64_t r, int64_t k, int64_t K)
+{
+    const int64_t q = k >> 7;
+    const int bb = (int)((k >> 4) & 7), t = (int)((k >> 2) & 3), n4 = (int)(k & 3);
+    int idx = 0;
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) {
+        int word, pos;
+        lut_locate<BITS>(bb, n4, b, word, pos);
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, q, t, word, K, BITS));
+        idx |= (int)((w >> pos) & 1u) << b;
+    }
+    return idx;
+}
+
+template <int BITS>
+__global__ void export_lut_kernel(const PackedHeader *hdr, const uint8_t *lut, int64_t N,
+                                  int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out)
 {
     const int64_t nw = K / 32;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0 && s_out) *s_out = hdr->s;
     if (i >= N * nw) return;
     const int64_t r = i / nw, j = i % nw;
-    uint32_t wd[3];
+    uint32_t c[BITS];
 #pragma unroll
-    for (int p = 0; p < 3; ++p) wd[p] = *reinterpret_cast<const uint32_t *>(lut + lut_word_offset(r, j, p, K));
+    for (int p = 0; p < BITS; ++p) c[p] = 0u;
+    for (int e = 0; e < 32; ++e) {
+        const int idx = lut_read_index<BITS>(lut, r, j * 32 + e, K);
 #pragma unroll
-    for (int p = 0; p < 3; ++p) {
-        uint32_t c = 0;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            int word, pos;
-            lut3_locate(p, i, word, pos);
-            c |= ((wd[word] >> pos) & 1u) << i;                                      // canonical: LSB-first bit-planes
-        }
-        planes_out[(r * 3 + p) * nw + j] = c;
+        for (int p = 0; p < BITS; ++p) c[p] |= (uint32_t)((idx >> p) & 1) << e;      // canonical: LSB-first bit-planes
     }
-    scales_out[r * (K / 16) + 2 * j] = lut[lut_scale_offset(r, 2 * j, K)];
-    scales_out[r * (K / 16) + 2 * j + 1] = lut[lut_scale_offset(r, 2 * j + 1, K)];
+#pragma unroll
+    for (int p = 0; p < BITS; ++p) planes_out[(r * BITS + p) * nw + j] = c[p];
+    scales_out[r * (K / 16) + 2 * j] = lut[lut_scale_offset(r, 2 * j, K, BITS)];
+    scales_out[r * (K / 16) + 2 * j + 1] = lut[lut_scale_offset(r, 2 * j + 1, K, BITS)];
 }
 
-cudaError_t launch_export_lut3(const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
-                               int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
-                               cudaStream_t stream)
+cudaError_t launch_export_lut(int bits, const PackedHeader *hdr, const uint8_t *lut_dev, int64_t N,
+                              int64_t K, uint32_t *planes_out, uint8_t *scales_out, float *s_out,
+                              cudaStream_t stream)
 {
     const int64_t total = N * (K / 32);
-    export_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(hdr, lut_dev, N, K, planes_out,
-                                                                            scales_out, s_out);
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (bits == 3) export_lut_kernel<3><<<blocks, 256, 0, stream>>>(hdr, lut_dev, N, K, planes_out, scales_out, s_out);
+    else export_lut_kernel<2><<<blocks, 256, 0, stream>>>(hdr, lut_dev, N, K, planes_out, scales_out, s_out);
     return cudaGetLastError();
 }
 
@@ -417,28 +461,41 @@ __global__ void import_nvfp4_kernel(const uint8_t *codes_in, const uint8_t *scal
     sf[sf_swizzled_offset(r, b, K)] = scales_in[r * nb + b];
 }
 
-__global__ void import_lut3_kernel(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
-                                   uint8_t *lut)
+// one thread per word group, as in the packer
+template <int BITS>
+__global__ void import_lut_kernel(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                                  uint8_t *lut)
 {
-    const int64_t nw = K / 32;
+    const int64_t nq = K / 128, nw = K / 32;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N * nw) return;
-    const int64_t r = i / nw, j = i % nw;
-    uint32_t wd[3] = {0u, 0u, 0u};
+    const int64_t quad = i >> 2;
+    const int t = (int)(i & 3);
+    if (quad >= N * nq) return;
+    const int64_t r = quad / nq, q = quad % nq;
+    uint32_t wd[BITS];
 #pragma unroll
-    for (int p = 0; p < 3; ++p) {
-        const uint32_t c = planes_in[(r * 3 + p) * nw + j];                        // canonical: LSB-first bit-planes
+    for (int p = 0; p < BITS; ++p) wd[p] = 0u;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            int word, pos;
-            lut3_locate(p, i, word, pos);
-            wd[word] |= ((c >> i) & 1u) << pos;
-        }
+    for (int bb = 0; bb < 8; ++bb) {
+        // weights 16 bb + 4 t .. + 3 of the 128: bits 16 (bb % 2) + 4 t .. of canonical word 4 q + bb / 2
+        uint32_t c[BITS];
+#pragma unroll
+        for (int p = 0; p < BITS; ++p) c[p] = planes_in[(r * BITS + p) * nw + q * 4 + (bb >> 1)] >> (16 * (bb & 1) + 4 * t);
+#pragma unroll
+        for (int n4 = 0; n4 < 4; ++n4)
+#pragma unroll
+            for (int b = 0; b < BITS; ++b) {
+                int word, pos;
+                lut_locate<BITS>(bb, n4, b, word, pos);
+                wd[word] |= ((c[b] >> n4) & 1u) << pos;
+            }
     }
 #pragma unroll
-    for (int p = 0; p < 3; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, j, p, K)) = wd[p];
-    lut[lut_scale_offset(r, 2 * j, K)] = scales_in[r * (K / 16) + 2 * j];
-    lut[lut_scale_offset(r, 2 * j + 1, K)] = scales_in[r * (K / 16) + 2 * j + 1];
+    for (int p = 0; p < BITS; ++p) *reinterpret_cast<uint32_t *>(lut + lut_word_offset(r, q, t, p, K, BITS)) = wd[p];
+    if (t == 0) {
+#pragma unroll
+        for (int bb = 0; bb < 8; ++bb) lut[lut_scale_offset(r, q * 8 + bb, K, BITS)] = scales_in[r * (K / 16) + q * 8 + bb];
+    }
 }
 
 __global__ void set_scale_kernel(PackedHeader *hdr, float s)
@@ -464,11 +521,13 @@ cudaError_t launch_import_nvfp4(const uint8_t *codes_in, const uint8_t *scales_i
     return cudaGetLastError();
 }
 
-cudaError_t launch_import_lut3(const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
-                               uint8_t *lut_dev, cudaStream_t stream)
+cudaError_t launch_import_lut(int bits, const uint32_t *planes_in, const uint8_t *scales_in, int64_t N, int64_t K,
+                              uint8_t *lut_dev, cudaStream_t stream)
 {
-    const int64_t total = N * (K / 32);
-    import_lut3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(planes_in, scales_in, N, K, lut_dev);
+    const int64_t total = N * (K / 128) * 4;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (bits == 3) import_lut_kernel<3><<<blocks, 256, 0, stream>>>(planes_in, scales_in, N, K, lut_dev);
+    else import_lut_kernel<2><<<blocks, 256, 0, stream>>>(planes_in, scales_in, N, K, lut_dev);
     return cudaGetLastError();
 }
 

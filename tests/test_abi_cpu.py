@@ -31,14 +31,29 @@ def test_library_exports_every_declared_symbol(dq):
     assert dq.status_string(0) == "ok" and "shape" in dq.status_string(2)
 
 
+def test_library_exports_nothing_the_header_does_not_declare(dq):
+    """Every dynamic symbol named dq_* of libdq.so is declared in include/dq.h (no hidden switches)."""
+    import subprocess
+    header = (ROOT / "include" / "dq.h").read_text()
+    declared = set(re.findall(r"\b(dq_[a-z0-9_]+)\s*\(", header))
+    from paper_2609_26333_b200 import binding
+    out = subprocess.run(["nm", "-D", "--defined-only", str(binding._LIB_PATH)], capture_output=True, text=True, check=True).stdout
+    exported = {line.split()[-1] for line in out.splitlines() if line.split() and line.split()[-1].startswith("dq_")}
+    assert exported, "nm listed no dq_* symbol"
+    assert exported <= declared, sorted(exported - declared)
+
+
 def test_packed_bytes_follows_storage_cost(dq):
     N, K = 6144, 4096
     nv = dq.packed_bytes(N, K, dq.FMT_NVFP4) - 1024
-    lut = dq.packed_bytes(N, K, dq.FMT_LUT3) - 1024 - 65536      # header + the decode kernel's 64 KiB lookup table
+    lut = dq.packed_bytes(N, K, dq.FMT_LUT3) - 1024
+    lut2 = dq.packed_bytes(N, K, dq.FMT_LUT2) - 1024
     assert nv == N * K // 2 + N * K // 16           # 4.5 bit per weight
     assert lut == 3 * N * K // 8 + N * K // 16      # 3.5 bit per weight
-    assert dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3) == 1024 + 65536 + nv + lut
-    assert dq.packed_bytes(N, K, dq.FMT_NVFP4_FROM_LUT3) == 1024 + 65536 + nv + lut
+    assert lut2 == 2 * N * K // 8 + N * K // 16     # 2.5 bit per weight
+    assert dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3) == 1024 + nv + lut
+    assert dq.packed_bytes(N, K, dq.FMT_NVFP4_FROM_LUT3) == 1024 + nv + lut
+    assert dq.packed_bytes(N, K, dq.FMT_LUT3 | dq.FMT_LUT2) == 1024 + lut + lut2
 
 
 def test_argument_validation_needs_no_device(dq):
@@ -49,6 +64,10 @@ def test_argument_validation_needs_no_device(dq):
     assert L.dq_packed_bytes(512, 256, 0, C.byref(out)) == 1          # no format
     assert L.dq_packed_bytes(512, 256, 1 | 4, C.byref(out)) == 1      # two NVFP4 views
     assert L.dq_packed_bytes(512, 256, 3, None) == 1
+    assert L.dq_packed_bytes(512, 32768 + 128, 1, C.byref(out)) == 0  # NVFP4 alone has no K limit
+    assert L.dq_packed_bytes(512, 32768 + 128, 2, C.byref(out)) == 2  # LUT decode keeps a row of K in shared memory
+    assert L.dq_packed_bytes(512, 32768 + 128, 8, C.byref(out)) == 2
+    assert L.dq_packed_bytes(512, 256, 16, C.byref(out)) == 1         # unknown format bit
     h = C.c_void_p(0)
     assert L.dq_pack_weights(None, 0, 512, 256, 256, 3, None, None, 0, None, C.byref(h)) == 1
     assert L.dq_pack_weights(4096, 7, 512, 256, 256, 3, None, 4096, 1 << 20, None, C.byref(h)) == 1   # dtype
@@ -60,6 +79,8 @@ def test_argument_validation_needs_no_device(dq):
     assert L.dq_free_weights(None) == 1
     assert L.dq_prefill_linear(None, 4096, 1, 256, 1.0, 4096, 512, 4096, 0, None) == 1
     assert L.dq_decode_linear(None, 4096, 1, 256, 4096, 512, None) == 1
+    assert L.dq_decode_linear_lut2(None, 4096, 1, 256, 4096, 512, None) == 1
+    assert L.dq_test_decode_linear(None, 2, 0, 0, 0, 0, 0, 4096, 1, 256, 4096, 512, None) == 1
     assert L.dq_quantize_activations(4096, 4, 200, 200, 1.0, 4096, 4096, None) == 2
     assert L.dq_quantize_activations(4096, 4, 256, 256, 0.0, 4096, 4096, None) == 1
     assert L.dq_quantize_activations(4096, 4, 256, 256, float("nan"), 4096, 4096, None) == 1

@@ -313,35 +313,56 @@ def test_decode_nvfp4_kernels_agree_and_handle_wide_range_activations(dq, oracle
     g = torch.Generator().manual_seed(91)
     X = (torch.randn(B, K, generator=g) * torch.exp2(torch.randint(-20, 12, (B, K), generator=g).float())).to(torch.bfloat16)
     Yr, S = oracle.decode_linear_nvfp4(dq_inputs.bf16_to_f32_numpy(X), ref["nvfp4_codes"], ref["nvfp4_scales"], ref["s"])
-    for which in (1, 0):
-        old = dq.lib().dq_debug_nvfp4_decode_kernel(which)
-        try:
-            out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
-            dq.decode_linear_nvfp4(w, X.to(DEV), out=out[:, :N])
-            _status_ok(dq)
-        finally:
-            dq.lib().dq_debug_nvfp4_decode_kernel(old)
+    for variant in (0, 1):
+        out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+        dq.test_decode_linear(w, dq.FMT_NVFP4, X.to(DEV), out=out[:, :N], variant=variant)
+        _status_ok(dq)
         assert torch.all(out[:, N:] == -3.0)
-        check_outputs(_f64(out[:, :N]), Yr, S, f"nvfp4 decode kernel {which}, wide-range activations")
+        check_outputs(_f64(out[:, :N]), Yr, S, f"nvfp4 decode kernel variant {variant}, wide-range activations")
 
 
-@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(272, 17408, 33)])
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(272, 17408, 33), (48, 32768, 34)])
 @pytest.mark.parametrize("B", [1, 3, 8, 11])
-def test_decode_lut3_tensor_core_kernel_parity(dq, oracle, N, K, seed, B):
-    """The tensor-core LUT3 kernel (the batch >= 3 path), forced for every batch size here."""
+def test_decode_lut3_long_rows_and_forced_work_splits(dq, oracle, N, K, seed, B):
+    """Default launch on long rows, then the same call with other splits of the work: one warp per tile, many
+    warps per tile (several slices or a single atom each), shallow and deep copy rings."""
     W, ref = _layer(oracle, N, K, seed)
     w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
     X = dq_inputs.gaussian_bf16(B, K, 1.0, 2000 + seed + B)
-    old = dq.lib().dq_debug_lut3_decode_kernel(1)
-    try:
-        out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
-        dq.decode_linear(w, X.to(DEV), out=out[:, :N])
-        _status_ok(dq)
-    finally:
-        dq.lib().dq_debug_lut3_decode_kernel(old)
-    assert torch.all(out[:, N:] == -3.0)
     Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
-    check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 tensor-core decode {B}x{N}x{K}")
+    out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+    dq.decode_linear(w, X.to(DEV), out=out[:, :N])
+    _status_ok(dq)
+    assert torch.all(out[:, N:] == -3.0)
+    check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 decode {B}x{N}x{K}")
+    if B in (1, 3):
+        slices = (K + 1023) // 1024
+        for P, G, S_ in ((1, 1, 2), (1, 7, 3), (min(slices, 3), 2, 8), (min(slices, 16), 1, 4), (min(slices, 32), 1, 2)):
+            if 4096 + P * G * (512 + 1152 + S_ * 3584) + (slices * 2048 + 16) > 227 * 1024:
+                continue                                     # does not fit shared memory even with one column per pass
+            got = dq.test_decode_linear(w, dq.FMT_LUT3, X.to(DEV), warps_per_group=P, groups_per_cta=G, ring_stages=S_)
+            _status_ok(dq)
+            check_outputs(_f64(got), Yr, S, f"lut3 decode {B}x{N}x{K}, split P={P} G={G} S={S_}")
+
+
+def test_decode_wait_budget_runs_out_cleanly(dq, oracle):
+    """A device-side wait that gives up: one bulk copy is never requested (test hook), the wait for it runs out
+    after a millisecond, the kernel returns normally, the status word says DQ_ERR_TIMEOUT, and the next call is right."""
+    N, K = 4096, 4096
+    W, ref = _layer(oracle, N, K, 99)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    X = dq_inputs.gaussian_bf16(2, K, 1.0, 100).to(DEV)
+    torch.cuda.synchronize()
+    assert dq.get_status()[0] == 0
+    dq.test_decode_linear(w, dq.FMT_LUT3, X, variant=1, wait_cycles=2_000_000)
+    torch.cuda.synchronize()
+    st, det = dq.get_status()
+    assert st == 7 and (det & 0xFF000) == 0x36000, (st, hex(det))      # DQ_ERR_TIMEOUT from the LUT decode kernel
+    assert dq.get_status()[0] == 0                                     # the read cleared it
+    Y = dq.decode_linear(w, X)
+    _status_ok(dq)
+    Yr, S = oracle.decode_linear(dq_inputs.bf16_to_f32_numpy(X.cpu()), ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    check_outputs(_f64(Y), Yr, S, "decode after a timed-out call")
 
 
 def _sparse_patterns(K, seed):
