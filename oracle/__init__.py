@@ -72,6 +72,12 @@ def lib() -> ctypes.CDLL:
         L.dqo_quant_nvfp4.argtypes = [f32p, i64, i64, i64, c.c_float, u8p, u8p]
         L.dqo_quant_lut3.restype = None
         L.dqo_quant_lut3.argtypes = [f32p, i64, i64, i64, c.c_float, u16p, u32p, u8p]
+        L.dqo_lut2_default_codebook.restype = None
+        L.dqo_lut2_default_codebook.argtypes = [u16p]
+        L.dqo_quant_lut2.restype = None
+        L.dqo_quant_lut2.argtypes = [f32p, i64, i64, i64, c.c_float, u16p, u32p, u8p]
+        L.dqo_dequant_lut2.restype = None
+        L.dqo_dequant_lut2.argtypes = [u32p, u8p, i64, i64, c.c_float, u16p, f64p]
         L.dqo_autocast_lut3_to_nvfp4.restype = None
         L.dqo_autocast_lut3_to_nvfp4.argtypes = [u32p, u8p, i64, i64, u16p, u8p, u8p]
         L.dqo_dequant_nvfp4.restype = None
@@ -139,6 +145,13 @@ def lut3_default_codebook() -> np.ndarray:
     return cb
 
 
+def lut2_default_codebook() -> np.ndarray:
+    """The LUT2A16 grid of App. A.3 rounded to fp16, as uint16 bit patterns."""
+    cb = np.zeros(4, dtype=np.uint16)
+    lib().dqo_lut2_default_codebook(_p(cb, ctypes.c_uint16))
+    return cb
+
+
 def codebook_values(codebook_f16: np.ndarray) -> np.ndarray:
     return np.array([f16_decode(int(h)) for h in codebook_f16], dtype=np.float64)
 
@@ -186,6 +199,21 @@ def quant_lut3(x, s: float, codebook_f16=None):
     return planes, scales
 
 
+def quant_lut2(x, s: float, codebook_f16=None):
+    """RTN LUT2 of a (rows, K) fp32 matrix (App. A.3 "LUT formats", 4 levels).
+
+    Returns (planes uint32[rows, 2, K/32], scales uint8[rows, K/16] signed E4M3)."""
+    x = _f32_2d(x)
+    rows, K = x.shape
+    assert K % 32 == 0
+    cb = lut2_default_codebook() if codebook_f16 is None else np.ascontiguousarray(codebook_f16, dtype=np.uint16)
+    planes = np.zeros((rows, 2, K // 32), dtype=np.uint32)
+    scales = np.zeros((rows, K // BLOCK), dtype=np.uint8)
+    lib().dqo_quant_lut2(_p(x, ctypes.c_float), rows, K, K, np.float32(s), _p(cb, ctypes.c_uint16),
+                         _p(planes, ctypes.c_uint32), _p(scales, ctypes.c_uint8))
+    return planes, scales
+
+
 def autocast_lut3_to_nvfp4(planes, lut_scales, codebook_f16=None):
     """NVFP4 view of LUT3 weights (Sec. 2.3 autocast). Returns (codes, scales)."""
     planes = np.ascontiguousarray(planes, dtype=np.uint32)
@@ -221,6 +249,26 @@ def dequant_lut3(planes, scales, s: float, codebook_f16=None) -> np.ndarray:
     lib().dqo_dequant_lut3(_p(planes, ctypes.c_uint32), _p(scales, ctypes.c_uint8), rows, K, np.float32(s),
                            _p(cb, ctypes.c_uint16), _p(out, ctypes.c_double))
     return out
+
+
+def dequant_lut2(planes, scales, s: float, codebook_f16=None) -> np.ndarray:
+    planes = np.ascontiguousarray(planes, dtype=np.uint32)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    rows, K = planes.shape[0], planes.shape[2] * 32
+    cb = lut2_default_codebook() if codebook_f16 is None else np.ascontiguousarray(codebook_f16, dtype=np.uint16)
+    out = np.zeros((rows, K), dtype=np.float64)
+    lib().dqo_dequant_lut2(_p(planes, ctypes.c_uint32), _p(scales, ctypes.c_uint8), rows, K, np.float32(s),
+                           _p(cb, ctypes.c_uint16), _p(out, ctypes.c_double))
+    return out
+
+
+def unpack_lut2_indices(planes) -> np.ndarray:
+    """Bit-planes (rows, 2, K/32) -> indices (rows, K), LSB-first (App. C.2 storage)."""
+    planes = np.asarray(planes, dtype=np.uint32)
+    rows, _, W = planes.shape
+    bits = (planes[:, :, :, None] >> np.arange(32, dtype=np.uint32)) & 1      # rows,2,W,32
+    idx = bits[:, 0] | (bits[:, 1] << 1)
+    return idx.reshape(rows, W * 32).astype(np.uint8)
 
 
 def unpack_lut3_indices(planes) -> np.ndarray:
@@ -290,6 +338,13 @@ def decode_linear_nvfp4(X_f32, nv_codes, nv_scales, s_w: float, lib_matmul=True)
     times NVFP4-dequantised weights, fp64."""
     X = np.asarray(X_f32, dtype=np.float64)
     Wh = dequant_nvfp4(nv_codes, nv_scales, s_w)
+    return matmul_nt_lib(X, Wh) if lib_matmul else matmul_nt(X, Wh)
+
+
+def decode_linear_lut2(X_f32, planes, lut_scales, s_w: float, codebook_f16=None, lib_matmul=True):
+    """Decode: raw bf16 activations times LUT2-dequantised weights, fp64 (App. C.2, Table 1 LUT2 rows)."""
+    X = np.asarray(X_f32, dtype=np.float64)
+    Wh = dequant_lut2(planes, lut_scales, s_w, codebook_f16)
     return matmul_nt_lib(X, Wh) if lib_matmul else matmul_nt(X, Wh)
 
 

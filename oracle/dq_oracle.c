@@ -18,6 +18,7 @@
  *        block's maximum-magnitude element, so that element normalises to +6;
  *        element index = nearest level of the 8-level grid; indices stored
  *        bit-planed as int32 over (N, 3, K/32) (App. C.2).
+ *      LUT2 (same passage): the same rule with the 4-level grid, 2 bit-planes.
  *   4. autocast LUT3 -> NVFP4 (Sec. 2.3): re-quantise the LUT3 weights to NVFP4.
  *   5. dequantise x^ = s * d_b * level and fp64 products  Y = A^ W^T.
  *
@@ -186,6 +187,14 @@ void dqo_lut3_default_codebook(uint16_t codebook_f16[8])
     for (int j = 0; j < 8; ++j) codebook_f16[j] = dqo_f16_encode(DQO_LUT3_PAPER_GRID[j]);
 }
 
+/* The paper's LUT2A16 grid (App. A.3 "LUT formats": 4 levels, 2.5 bit per weight), rounded to fp16. */
+static const float DQO_LUT2_PAPER_GRID[4] = { -3.6517f, 0.0f, 2.5227f, 6.0f };
+
+void dqo_lut2_default_codebook(uint16_t codebook_f16[4])
+{
+    for (int j = 0; j < 4; ++j) codebook_f16[j] = dqo_f16_encode(DQO_LUT2_PAPER_GRID[j]);
+}
+
 /* ----------------------------------------------------------- global scale */
 
 /* App. A.3: s = max|W| / (6*448); fused layers pass the concatenated matrix. */
@@ -294,6 +303,55 @@ void dqo_quant_lut3(const float *x, int64_t rows, int64_t K, int64_t ld, float s
     }
 }
 
+/* LUT2 round-to-nearest (App. A.3 "LUT formats"; K % 32 == 0): the same rule as LUT3 with the
+ * 4-level grid -- signed block scale from the block's maximum-magnitude element (so that element
+ * normalises to +6), nearest level, a value exactly halfway goes to the lower level.
+ *   codebook_f16 : 4 fp16 levels, strictly increasing, containing 0 and 6
+ *   planes : uint32[rows][2][K/32] bit-planes (App. C.2 storage with b = 2)
+ *   scales : uint8[rows][K/16] signed E4M3, zero stored as 0x00            */
+void dqo_quant_lut2(const float *x, int64_t rows, int64_t K, int64_t ld, float s,
+                    const uint16_t codebook_f16[4], uint32_t *planes, uint8_t *scales)
+{
+    float G[4], T[3];
+    int zero_idx = 0;
+    for (int j = 0; j < 4; ++j) {
+        G[j] = dqo_f16_decode(codebook_f16[j]);
+        if (G[j] == 0.0f) zero_idx = j;
+    }
+    for (int j = 0; j < 3; ++j) T[j] = (G[j] + G[j + 1]) * 0.5f;   /* exact in fp32 */
+    const float rc6 = 1.0f / (6.0f * s);
+    const int64_t W = K / 32;
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        uint32_t *pl = planes + r * 2 * W;
+        for (int64_t j = 0; j < 2 * W; ++j) pl[j] = 0;
+        for (int64_t b = 0; b < K / DQO_BLOCK; ++b) {
+            const float *xb = x + r * ld + b * DQO_BLOCK;
+            float m = xb[0];
+            for (int i = 1; i < DQO_BLOCK; ++i) {
+                float v = xb[i];
+                if (fabsf(v) > fabsf(m) || (fabsf(v) == fabsf(m) && v > m)) m = v;
+            }
+            float t = m * rc6;
+            uint8_t d = dqo_e4m3_encode(t);
+            if ((d & 0x7F) == 0) d = 0;
+            scales[r * (K / DQO_BLOCK) + b] = d;
+            for (int i = 0; i < DQO_BLOCK; ++i) {
+                int idx = zero_idx;
+                if (d != 0) {
+                    float rr = 1.0f / (s * dqo_e4m3_decode(d));
+                    float y = xb[i] * rr;
+                    idx = 0;
+                    for (int j = 0; j < 3; ++j) idx += (y > T[j]);
+                }
+                int64_t k = b * DQO_BLOCK + i;
+                for (int p = 0; p < 2; ++p)
+                    pl[p * W + k / 32] |= (uint32_t)((idx >> p) & 1) << (k % 32);
+            }
+        }
+    }
+}
+
 /* Sec. 2.3 autocast: the NVFP4 view of LUT3 weights.  Each level maps to its
  * nearest E2M1 value; a negative block scale flips the element signs and the
  * NVFP4 block scale is |d_b| (the LUT3 block extreme is exactly 6*|d_b|*s, so
@@ -352,6 +410,21 @@ void dqo_dequant_lut3(const uint32_t *planes, const uint8_t *scales, int64_t row
             int idx = 0;
             for (int p = 0; p < 3; ++p)
                 idx |= (int)((planes[(r * 3 + p) * W + k / 32] >> (k % 32)) & 1u) << p;
+            double d = (double)dqo_e4m3_decode(scales[r * (K / DQO_BLOCK) + k / DQO_BLOCK]);
+            out[r * K + k] = (double)s * d * (double)dqo_f16_decode(codebook_f16[idx]);
+        }
+}
+
+void dqo_dequant_lut2(const uint32_t *planes, const uint8_t *scales, int64_t rows, int64_t K,
+                      float s, const uint16_t codebook_f16[4], double *out)
+{
+    const int64_t W = K / 32;
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            int idx = 0;
+            for (int p = 0; p < 2; ++p)
+                idx |= (int)((planes[(r * 2 + p) * W + k / 32] >> (k % 32)) & 1u) << p;
             double d = (double)dqo_e4m3_decode(scales[r * (K / DQO_BLOCK) + k / DQO_BLOCK]);
             out[r * K + k] = (double)s * d * (double)dqo_f16_decode(codebook_f16[idx]);
         }
