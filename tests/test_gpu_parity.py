@@ -434,6 +434,78 @@ def test_decode_lut3_wide_range_activations(dq, oracle):
         check_outputs(_f64(out[:, :N]), Yr, S, f"lut3 decode, wide-range activations, batch {B}")
 
 
+_lut2_cache = {}
+
+
+def _lut2_layer(oracle, N, K, seed):
+    key = (N, K, seed)
+    if key not in _lut2_cache:
+        W = dq_inputs.gaussian_bf16(N, K, 0.02, seed)
+        Wf = dq_inputs.bf16_to_f32_numpy(W)
+        s = oracle.global_scale(oracle.absmax(Wf))
+        _lut2_cache[key] = (W, s) + oracle.quant_lut2(Wf, s)
+    return _lut2_cache[key]
+
+
+@pytest.mark.parametrize("N,K,seed", [(512, 256, 0), (144, 384, 31), (784, 1152, 32)])
+def test_pack_lut2_bit_exact(dq, oracle, N, K, seed):
+    """LUT2 planes and signed scales against the oracle, alone and next to LUT3 in one handle."""
+    W, s, planes, scales = _lut2_layer(oracle, N, K, seed)
+    for fmts in (dq.FMT_LUT2, dq.FMT_LUT2 | dq.FMT_LUT3 | dq.FMT_NVFP4):
+        w = dq.pack_weights(W.to(DEV), formats=fmts)
+        p, sc, s_dev = dq.export_canonical(w, dq.FMT_LUT2)
+        _status_ok(dq)
+        assert np.float32(_np(s_dev)[0]) == np.float32(s)
+        assert _np(p).shape == (N, 2, K // 32)
+        assert np.array_equal(_np(sc), scales)
+        assert np.array_equal(_np(p).view(np.uint32), planes)
+    if fmts & dq.FMT_LUT3:
+        _, ref = _layer(oracle, N, K, seed)
+        p3, sc3, _ = dq.export_canonical(w, dq.FMT_LUT3)
+        assert np.array_equal(_np(p3).view(np.uint32), ref["lut3_planes"]) and np.array_equal(_np(sc3), ref["lut3_scales"])
+    # degenerate blocks: zeros, sign ties, one huge outlier
+    X = dq_inputs.gaussian_bf16(32, 128, 0.02, 34)
+    X[0, :16] = 0
+    X[1, 0], X[1, 5] = 0.5, -0.5
+    X[3, 7] = 3.0e4
+    Xf = dq_inputs.bf16_to_f32_numpy(X)
+    s2 = oracle.global_scale(oracle.absmax(Xf))
+    rp, rs = oracle.quant_lut2(Xf, s2)
+    p, sc, _ = dq.export_canonical(dq.pack_weights(X.to(DEV), formats=dq.FMT_LUT2), dq.FMT_LUT2)
+    assert np.array_equal(_np(p).view(np.uint32), rp) and np.array_equal(_np(sc), rs)
+
+
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(272, 17408, 33)])
+@pytest.mark.parametrize("B", [1, 2, 3, 8, 17, 64])
+def test_decode_lut2_parity(dq, oracle, N, K, seed, B):
+    W, s, planes, scales = _lut2_layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT2)
+    X = dq_inputs.gaussian_bf16(B, K, 1.0, 3000 + seed + B)
+    out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+    dq.decode_linear_lut2(w, X.to(DEV), out=out[:, :N])
+    _status_ok(dq)
+    assert torch.all(out[:, N:] == -3.0)
+    Yr, S = oracle.decode_linear_lut2(dq_inputs.bf16_to_f32_numpy(X), planes, scales, s)
+    check_outputs(_f64(out[:, :N]), Yr, S, f"lut2 decode {B}x{N}x{K}")
+
+
+def test_decode_lut2_sparse_activations_and_wrong_handle(dq, oracle):
+    N, K = 1024, 4096
+    W, s, planes, scales = _lut2_layer(oracle, N, K, 96)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT2)
+    P = _sparse_patterns(K, 97)
+    Yr, S = oracle.decode_linear_lut2(dq_inputs.bf16_to_f32_numpy(P), planes, scales, s)
+    for B in (1, 4):
+        got = torch.cat([dq.decode_linear_lut2(w, P.to(DEV)[i:i + B]) for i in range(0, P.shape[0], B)])
+        _status_ok(dq)
+        check_outputs(_f64(got), Yr, S, f"lut2 decode, sparse / cancelling activations, batch {B}")
+    with pytest.raises(dq.DQError):
+        dq.decode_linear(w, P.to(DEV)[:1])                        # no LUT3 in this handle
+    w3 = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    with pytest.raises(dq.DQError):
+        dq.decode_linear_lut2(w3, P.to(DEV)[:1])
+
+
 def test_decode_one_hot_and_strided(dq, oracle):
     N, K = 256, 512
     W, ref = _layer(oracle, N, K, 64)
