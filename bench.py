@@ -34,13 +34,15 @@ METRIC = "NVFP4 prefill GEMM TFLOP/s & LUT3 decode GEMV GB/s, % of B200 roofline
 DEFAULT_WORKLOAD = "c3_gate_up27b"
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum);
-# see profiles/ for the captures these come from.  None = not captured for that workload.
+# DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the kernel named in the
+# roofline object of the same line.  None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {
-    ("gemm", "c3_gate_up27b"): 79.2e6 + 240.4e6,      # profiles/launch_list_c3_gate_up27b.md
-    ("gemv", "c3_gate_up27b"): 39.10e6,
-    ("gemv_nvfp4", "c3_gate_up27b"): 50.2e6,          # profiles/gemv_nvfp4_mma_8192x4096.md (scaled by N x K)
+    ("gemm", "c3_gate_up27b"): 79.2e6 + 240.4e6,      # gemm_nvfp4_pair_kernel, full size
+    ("gemv", "c3_gate_up27b"): 39.04e6,               # gemv_lut_kernel<3, 384, 2>, full size, batch 1 (reads; writes are 35 KB)
+    ("gemv_nvfp4", "c3_gate_up27b"): 50.2e6,          # gemv_nvfp4_mma_kernel, small case scaled by N x K
 }
+NOMINAL_FP4_TFLOPS = 9000.0                            # dense FP4, 4 x the 2250 TFLOP/s bf16 figure
+NOMINAL_HBM_GBS = 8000.0
 
 
 def load_peaks():
@@ -55,7 +57,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
 
-    def __init__(self, device_index: int, period_s: float = 0.01):
+    def __init__(self, device_index: int, period_s: float = 0.001):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -156,7 +158,8 @@ def run_reference(args, cfg):
     total = time.perf_counter() - t0
     tflops = 2.0 * rows * cfg.N * cfg.K * args.steps / tp / 1e12
     dec_bytes = 0.4375 * cfg.N * cfg.K + 2 * cfg.K + 2 * cfg.N + 4
-    sample = f"{rows} of {cfg.M} prefill rows (dequantise + fp64 matmul of the whole N x K layer) + 1 decode token per step"
+    sample = (f"{rows} of {cfg.M} prefill rows (oracle quantise + dequantise of activations and of the whole N x K layer, "
+              f"then numpy's fp64 dgemm: oracle.matmul_nt_lib) + 1 decode token per step")
     line = {
         "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
@@ -303,6 +306,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-b2b", action="store_true", help="skip the back-to-back decode loops (short profiling runs)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for N GPUs outside a launcher: start N ranks (one per GPU) of this same command
+        from paper_2609_26333_b200 import replicas
+        os.execvp(sys.executable, replicas.spawn_command(args.gpus, [str(Path(__file__).resolve())] + sys.argv[1:]))
     args.warmup = max(args.warmup, 3) if args.impl == "dq" else args.warmup
     if args.workload == "c4_stack27b":
         if args.impl == "reference":
@@ -349,7 +356,8 @@ def main():
     A = A_host.to(dev)
     X = X_host.to(dev)
 
-    packed_bytes = dq.packed_bytes(N, K, dq.FMT_NVFP4 | dq.FMT_LUT3)
+    FORMATS = dq.FMT_NVFP4 | dq.FMT_LUT3 | dq.FMT_LUT2
+    packed_bytes = dq.packed_bytes(N, K, FORMATS)
     copies = args.copies or max(2, int(np.ceil(2.5 * L2_BYTES / (0.4375 * N * K))))
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -357,7 +365,7 @@ def main():
     for c in range(copies):
         if c == 1:
             e0.record()
-        ws.append(dq.pack_weights(W))
+        ws.append(dq.pack_weights(W, formats=FORMATS))
         if c == 1:
             e1.record()
     torch.cuda.synchronize()
@@ -437,6 +445,45 @@ def main():
     b1.record()
     torch.cuda.synchronize()
     d_nv_ms = b0.elapsed_time(b1) / nb2b
+    # and on the LUT2 weights (2.5 bit per weight)
+    for i in range(copies):
+        dq.decode_linear_lut2(ws[i], X, out=Yd)
+    torch.cuda.synchronize()
+    b0.record()
+    for i in range(nb2b):
+        dq.decode_linear_lut2(ws[i % copies], X, out=Yd)
+    b1.record()
+    torch.cuda.synchronize()
+    d_l2_ms = b0.elapsed_time(b1) / nb2b
+
+    # ---- measured ceilings (outside the timed region): the GEMM kernel's MMA issue sequence alone, and a
+    #      read-only 128-bit streaming pass over the packed copies
+    fp4_probe_tflops = stream_read_gbs = None
+    if M > 128 and not args.no_b2b:
+        for _ in range(3):
+            dq.bench_gemm_mma_only(ws[0], M, Y, workspace)
+        torch.cuda.synchronize()
+        b0.record()
+        for _ in range(10):
+            dq.bench_gemm_mma_only(ws[0], M, Y, workspace)
+        b1.record()
+        torch.cuda.synchronize()
+        fp4_probe_tflops = 2.0 * M * N * K / (b0.elapsed_time(b1) / 10 * 1e-3) / 1e12
+    if not args.no_b2b:
+        scratch = torch.zeros(8, dtype=torch.uint8, device=dev)
+        bufs = [w.packed for w in ws]
+        for t in bufs:
+            dq.bench_stream_read(t[: t.numel() // 16 * 16], scratch)
+        torch.cuda.synchronize()
+        b0.record()
+        for t in bufs:
+            dq.bench_stream_read(t[: t.numel() // 16 * 16], scratch)
+        b1.record()
+        torch.cuda.synchronize()
+        stream_read_gbs = sum(t.numel() // 16 * 16 for t in bufs) / (b0.elapsed_time(b1) * 1e-3) / 1e9
+        st, det = dq.get_status()
+        if st != 0:
+            raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the measurement hooks")
 
     # ---- end to end: pinned host buffers, copies inside the timed region ----
     e2e = None
@@ -471,9 +518,9 @@ def main():
 
     # ---- max over ranks ----
     from paper_2609_26333_b200 import replicas
-    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms, d_b2b_ms, d_nv_ms = replicas.max_over_ranks(
+    total_ms, q_ms, g_ms, d_ms, e2e_p_ms, e2e_d_ms, d_b2b_ms, d_nv_ms, d_l2_ms = replicas.max_over_ranks(
         [total_ms, q_ms, g_ms, d_ms, e2e["prefill_ms"] if e2e else 0.0, e2e["decode_ms"] if e2e else 0.0, d_b2b_ms,
-         d_nv_ms], device=dev)
+         d_nv_ms, d_l2_ms], device=dev)
 
     flops = 2.0 * M * N * K
     dec_bytes = 0.4375 * N * K + 2.0 * B * K + 2.0 * B * N + 4
@@ -482,7 +529,12 @@ def main():
     gemm_tflops = flops / (g_ms * 1e-3) / 1e12
     decode_gbs = dec_bytes / (d_ms * 1e-3) / 1e9
     quant_gbs = quant_bytes / (q_ms * 1e-3) / 1e9
-    fp4_peak = 4.0 * peaks["bf16_sustained"]
+    # FP4 tensor peak "of measured": 4 x the measured bf16 cuBLAS rate (nominal ratio fp4 : bf16), the burst figure
+    # when the whole timed region is shorter than a second (the clocks never settle under the power cap in that
+    # time), the sustained figure otherwise
+    burst = total_ms < 1000.0
+    fp4_peak = 4.0 * (peaks["bf16_burst"] if burst else peaks["bf16_sustained"])
+    sm_mhz = clocks.get("sm_mhz")
 
     line = {
         "metric": METRIC, "value": prefill_tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -505,15 +557,27 @@ def main():
                             "value": world * (0.5625 * N * K + 2.0 * B * (K + N)) / (d_nv_ms * 1e-3) / 1e9,
                             "frac_of_measured_hbm": (0.5625 * N * K + 2.0 * B * (K + N)) / (d_nv_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "pack_ms": pack_ms,
-        "roofline": {"kernel": "gemm_nvfp4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
+        "roofline": {"kernel": "gemm_nvfp4_pair_kernel" if M > 128 else "gemm_nvfp4_kernel", "bound": "tensor",
+                     "achieved": gemm_tflops, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(("gemm", cfg.name)),
-                     "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_sustained']} TFLOP/s); "
-                                    f"nominal dense FP4 9000"},
-        "roofline_decode": {"kernel": "gemv_lut3_mma_kernel" if cfg.name == DEFAULT_WORKLOAD or B >= 2 else "gemv_lut3_kernel / gemv_lut3_mma_kernel (by shape)", "bound": "hbm", "achieved": decode_gbs,
+                     "peak_source": f"4 x {peaks['source']} bf16 cuBLAS, {'burst' if burst else 'sustained'} figure "
+                                    f"({peaks['bf16_burst'] if burst else peaks['bf16_sustained']} TFLOP/s): the timed region "
+                                    f"lasted {total_ms:.0f} ms",
+                     "frac_of_4x_burst_bf16": gemm_tflops / (4.0 * peaks["bf16_burst"]),
+                     "frac_of_4x_sustained_bf16": gemm_tflops / (4.0 * peaks["bf16_sustained"]),
+                     "frac_of_nominal_fp4": gemm_tflops / NOMINAL_FP4_TFLOPS,
+                     "fp4_probe_tflops": fp4_probe_tflops,
+                     "frac_of_probe": gemm_tflops / fp4_probe_tflops if fp4_probe_tflops else None,
+                     "gemm_ms_x_sm_mhz": g_ms * sm_mhz if sm_mhz else None},
+        "roofline_decode": {"kernel": "gemv_lut_kernel<3>", "bound": "hbm", "achieved": decode_gbs,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": decode_gbs / peaks["hbm_gbs"],
-                            "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)),
-                            "peak_source": f"{peaks['source']} copy bandwidth"},
+                            "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)) if B == 1 else None,
+                            "peak_source": f"{peaks['source']} copy bandwidth",
+                            "timing": "inside the step, between the GEMM and the next step's quantiser",
+                            "frac_of_nominal_8tbs": decode_gbs / NOMINAL_HBM_GBS,
+                            "stream_read_gbs": stream_read_gbs,
+                            "decode_ms_x_sm_mhz": d_ms * sm_mhz if sm_mhz else None},
     }
     nv_bytes = 0.5625 * N * K + 2.0 * B * (K + N)
     line["roofline_decode_nvfp4a16"] = {"kernel": "gemv_nvfp4_mma_kernel", "bound": "hbm",
@@ -522,7 +586,15 @@ def main():
                                         "traffic": NCU_TRAFFIC_BYTES.get(("gemv_nvfp4", cfg.name)),
                                         "timing": "back-to-back launches", "peak_source": f"{peaks['source']} copy bandwidth"}
     line["roofline_decode"]["back_to_back"] = {"achieved": dec_bytes / (d_b2b_ms * 1e-3) / 1e9,
-                                               "frac": dec_bytes / (d_b2b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                                               "frac": dec_bytes / (d_b2b_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                               "frac_of_stream_read": dec_bytes / (d_b2b_ms * 1e-3) / 1e9 / stream_read_gbs
+                                               if stream_read_gbs else None}
+    l2_bytes = 0.3125 * N * K + 2.0 * B * (K + N) + 4
+    line["roofline_decode_lut2"] = {"kernel": "gemv_lut_kernel<2>", "bound": "hbm", "achieved": l2_bytes / (d_l2_ms * 1e-3) / 1e9,
+                                    "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                    "frac": l2_bytes / (d_l2_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                                    "ms": d_l2_ms, "timing": "back-to-back launches",
+                                    "peak_source": f"{peaks['source']} copy bandwidth"}
     if e2e:
         line["e2e"] = {"value": world * flops / (e2e_p_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": int(2 * M * K + 2 * B * K), "d2h_bytes_per_step": int(2 * M * N + 2 * B * N),
@@ -547,8 +619,8 @@ def main():
         line["cpu_baseline"] = {"value": 2.0 * rows * N * K / tp / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
                                 "kind": "oracle",
                                 "sample": f"{passes} passes of {rows} of {M} prefill rows against the whole {N}x{K} layer "
-                                          f"(quantise + dequantise + fp64 matmul, {tp:.1f} s each) and 1 decode token "
-                                          f"({td:.1f} s each)",
+                                          f"(oracle quantise + dequantise, then numpy's fp64 dgemm (oracle.matmul_nt_lib), "
+                                          f"{tp:.1f} s each) and 1 decode token ({td:.1f} s each)",
                                 "decode_gbs": (0.4375 * N * K + 2 * K + 2 * N + 4) / td / 1e9}
     if rank == 0:
         print(json.dumps(line), flush=True)

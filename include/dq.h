@@ -297,6 +297,26 @@ int dq_test_decode_linear(const dq_weights *w, unsigned format, int variant, int
                           int groups_per_cta, int ring_stages, long long wait_cycles, const void *X_dev,
                           int64_t B, int64_t ldx, void *Y_dev, int64_t ldy, void *stream);
 
+/* ---- measurement hooks (the paper has no counterpart; they give bench.py its two measured ceilings) ---- */
+
+/*
+ * The prefill GEMM kernel reduced to its tensor-core instruction stream: same launch, roles and barriers as
+ * dq_prefill_gemm for M > 128, but no operand or scale loads, no scale copies and no stores (Y_dev is not
+ * written; the products are computed on whatever shared memory holds).  2*M*N*K divided by its time is the
+ * block-scaled FP4 rate this kernel's MMA sequence reaches on this GPU at the clock it runs at: the measured
+ * FP4 tensor peak the roofline fraction is quoted against beside the nominal figure.  M must exceed 128;
+ * arguments otherwise as dq_prefill_gemm (the workspace need not have been filled).
+ */
+int dq_bench_gemm_mma_only(const dq_weights *w, int64_t M, void *Y_dev, int64_t ldy,
+                           const void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
+ * Reads `bytes` bytes at src_dev once with 128-bit loads and nothing else (a grid of 4 CTAs per SM): bytes
+ * divided by its time is the practical read-only streaming ceiling for the decode kernels.  out_dev: 8 bytes
+ * of device memory (a counter that keeps the loads alive), src_dev 16-byte aligned.
+ */
+int dq_bench_stream_read(const void *src_dev, size_t bytes, void *out_dev, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

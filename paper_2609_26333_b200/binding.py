@@ -21,7 +21,8 @@ DT_FP32 = 1
 SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights", "dq_free_weights",
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
-           "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear", "dq_export_canonical", "dq_import_canonical",
+           "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear",
+           "dq_bench_gemm_mma_only", "dq_bench_stream_read", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
            "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
@@ -80,6 +81,10 @@ def lib() -> C.CDLL:
         L.dq_test_decode_linear.restype = C.c_int
         L.dq_test_decode_linear.argtypes = [vp, C.c_uint, C.c_int, C.c_int, C.c_int, C.c_int, C.c_longlong, vp, i64, i64,
                                             vp, i64, vp]
+        L.dq_bench_gemm_mma_only.restype = C.c_int
+        L.dq_bench_gemm_mma_only.argtypes = [vp, i64, vp, i64, vp, sz, vp]
+        L.dq_bench_stream_read.restype = C.c_int
+        L.dq_bench_stream_read.argtypes = [vp, sz, vp, vp]
         L.dq_import_canonical.restype = C.c_int
         L.dq_import_canonical.argtypes = [C.c_int64, C.c_int64, C.c_uint, vp, vp, vp, vp, C.c_float,
                                           C.POINTER(C.c_uint16), vp, C.c_size_t, vp, C.POINTER(vp)]
@@ -295,6 +300,18 @@ def test_decode_linear(w: DQWeights, fmt: int, X: torch.Tensor, out: torch.Tenso
 
 
 test_decode_linear.__test__ = False      # not a pytest test
+
+
+def bench_gemm_mma_only(w: DQWeights, M: int, out: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """dq_bench_gemm_mma_only: the GEMM kernel's MMA issue sequence alone (measurement hook; `out` is not written)."""
+    _check(lib().dq_bench_gemm_mma_only(w.handle, M, out.data_ptr(), out.stride(0), workspace.data_ptr(),
+                                        workspace.numel(), _stream_ptr(stream)), "dq_bench_gemm_mma_only")
+
+
+def bench_stream_read(src: torch.Tensor, scratch: torch.Tensor, stream=None):
+    """dq_bench_stream_read: read `src` once with 128-bit loads (measurement hook); scratch: >= 8 bytes on the device."""
+    _check(lib().dq_bench_stream_read(src.data_ptr(), src.numel() * src.element_size(), scratch.data_ptr(),
+                                      _stream_ptr(stream)), "dq_bench_stream_read")
 
 
 def prefill_host_staging_bytes(w: DQWeights, M: int) -> int:

@@ -349,13 +349,14 @@ int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64
     return DQ_OK;
 }
 
-int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
-                    const void *workspace_dev, size_t workspace_bytes, void *stream)
+static int prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
+                        const void *workspace_dev, size_t workspace_bytes, void *stream, bool mma_only)
 {
     if (!Y_dev) return DQ_ERR_INVALID_ARG;
     int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
     if (st != DQ_OK) return st;
     if (ldy < w->N || ldy % 8 != 0 || !aligned(Y_dev, 16)) return DQ_ERR_ALIGN;
+    if (mma_only && M <= 128) return DQ_ERR_INVALID_ARG;          // the measurement mode exists in the pair kernel only
     st = check_arch();
     if (st != DQ_OK) return st;
     dq::StatusWord *sw = status_word_ptr();
@@ -375,7 +376,31 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
     g.N = w->N;
     g.K = w->K;
     g.status = sw;
+    g.mma_only = mma_only;
     if (dq::launch_gemm_nvfp4(g, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
+                    const void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    return prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream, false);
+}
+
+int dq_bench_gemm_mma_only(const dq_weights *w, int64_t M, void *Y_dev, int64_t ldy, const void *workspace_dev,
+                           size_t workspace_bytes, void *stream)
+{
+    return prefill_gemm(w, M, 1.0f, Y_dev, ldy, workspace_dev, workspace_bytes, stream, true);
+}
+
+int dq_bench_stream_read(const void *src_dev, size_t bytes, void *out_dev, void *stream)
+{
+    if (!src_dev || !out_dev || bytes < 16) return DQ_ERR_INVALID_ARG;
+    if (!aligned(src_dev, 16) || !aligned(out_dev, 8)) return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    if (dq::launch_stream_read(src_dev, bytes, out_dev, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return DQ_ERR_CUDA;
     return DQ_OK;
 }
 

@@ -13,6 +13,7 @@
 namespace dq {
 
 constexpr int kBlock = 16;            // weights per block scale (App. A.3)
+constexpr int kMaxDevices = 64;       // per-device one-time set-up flags
 constexpr int kSfAtomRows = 128;      // rows of one scale-factor atom of the block-scaled MMA
 constexpr int kSfAtomBytes = 512;     // 128 rows x 4 scales (64 k)
 constexpr int kSfRowPad = 256;        // NVFP4 scale tiles padded to the GEMM's N tile
@@ -196,7 +197,7 @@ struct GemmArgs {
     void *Y; int64_t ldy;
     int64_t M, N, K;
     StatusWord *status;
-    int probe = 0;   // timing probes: 1 = no MMA, 2 = no loads, 4 = no scale copies (results are meaningless), 8 = force the 1-CTA kernel
+    bool mma_only = false;   // measurement: MMA issue sequence only (pair kernel; no loads, scale copies or stores)
 };
 cudaError_t launch_gemm_nvfp4(const GemmArgs &args, cudaStream_t stream);
 cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &args, void *encode_fn, cudaStream_t stream);
@@ -227,6 +228,8 @@ struct GemvNvArgs {
 };
 cudaError_t launch_gemv_nvfp4(const GemvNvArgs &args, cudaStream_t stream);          // CUDA cores, pair-table lookups
 cudaError_t launch_gemv_nvfp4_mma(const GemvNvArgs &args, cudaStream_t stream);      // tensor cores (mma.sync), no lookups
-cudaError_t launch_fill_e2m1_table(cudaStream_t stream);   // value-pair table of the NVFP4 decode kernel
+cudaError_t launch_fill_e2m1_table(cudaStream_t stream);
+// read-only streaming sum with 128-bit loads (measurement): 8 bytes of result at out_dev
+cudaError_t launch_stream_read(const void *src_dev, size_t bytes, void *out_dev, cudaStream_t stream);   // value-pair table of the NVFP4 decode kernel
 
 }  // namespace dq

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                   const uint8_t *__restrict__ a_sf, const uint8_t *__restrict__ w_sf,
                   const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y, int64_t ldy,
-                  int M, int N, int K, StatusWord *status, int probe)
+                  int M, int N, int K, StatusWord *status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -119,7 +119,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t sSFA = sB + B_STAGE_BYTES;
                     const uint32_t sSFB = sSFA + SFA_STAGE_BYTES;
                     const uint32_t sf_bytes = (uint32_t)nkb * 512u;
-                    if (probe & 2) { mbar_arrive(full_bar(stage)); if (++stage == kStages) { stage = 0; phase ^= 1u; } continue; }
                     mbar_expect_tx(full_bar(stage), A_STAGE_BYTES + B_STAGE_BYTES + 3u * sf_bytes);
                     tma_load_2d(sA, &tmap_a, ks * 128, mb * BM, full_bar(stage));
                     tma_load_2d(sB, &tmap_w, ks * 128, nb * BN, full_bar(stage));
@@ -152,14 +151,14 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t sSFB = sSFA + SFA_STAGE_BYTES;
                     const uint32_t t_sfa = tmem_base + kTmemSfBase + sfbuf * kTmemSfBufCols;
                     const uint32_t t_sfb = t_sfa + 16u;
-                    for (int kb = 0; kb < nkb && !(probe & 4); ++kb) {
+                    for (int kb = 0; kb < nkb; ++kb) {
                         tmem_cp_sf(t_sfa + 4u * kb, make_desc_sf(sSFA + 512u * kb));
                         tmem_cp_sf(t_sfb + 8u * kb, make_desc_sf(sSFB + 512u * kb));
                         tmem_cp_sf(t_sfb + 8u * kb + 4u, make_desc_sf(sSFB + kKbPerStage * 512u + 512u * kb));
                     }
                     const uint64_t adesc = make_desc_sw128(sA);
                     const uint64_t bdesc = make_desc_sw128(sB);
-                    for (int kb = 0; kb < nkb && !(probe & 1); ++kb) {
+                    for (int kb = 0; kb < nkb; ++kb) {
                         // one k-step is 64 elements = 32 bytes inside the 128-byte swizzle row
                         mma_nvf4(tmem_base, adesc + 2ull * kb, bdesc + 2ull * kb, kInstrDesc, t_sfa + 4u * kb,
                                  t_sfb + 8u * kb, (ks > 0 || kb > 0) ? 1u : 0u);
@@ -266,24 +265,25 @@ cudaError_t launch_gemm_nvfp4(const GemmArgs &a, cudaStream_t stream)
 {
     if (gemm_init_driver_api() != 0) return cudaErrorNotSupported;
     // more than one 128-row block: CTA pairs share the W tile; otherwise a lone CTA per tile
-    if (a.M > BM && !(a.probe & 8)) return launch_gemm_nvfp4_pair(a, reinterpret_cast<void *>(g_encode), stream);
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (a.M > BM) return launch_gemm_nvfp4_pair(a, reinterpret_cast<void *>(g_encode), stream);
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     CUtensorMap tmap_a, tmap_w;
     if (!make_codes_tmap(&tmap_a, a.a_codes, a.M, a.K, BM)) return cudaErrorInvalidValue;
     if (!make_codes_tmap(&tmap_w, a.w_codes, a.N, a.K, BN)) return cudaErrorInvalidValue;
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
+    int sms = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = (int)(((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN));
     const int grid = tiles < sms ? tiles : sms;
     gemm_nvfp4_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(tmap_a, tmap_w, a.a_sf, a.w_sf, a.hdr, a.act_scale,
                                                              reinterpret_cast<__nv_bfloat16 *>(a.Y), a.ldy, (int)a.M,
-                                                             (int)a.N, (int)a.K, a.status, a.probe);
+                                                             (int)a.N, (int)a.K, a.status);
     return cudaGetLastError();
 }
 

@@ -160,11 +160,15 @@ __device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, in
     nb = r / gsz;
 }
 
+// MMA_ONLY (measurement): the same roles and barriers, but no operand or scale loads (the barriers are completed by
+// hand), no scale copies into TMEM and no stores: what is left is the MMA issue sequence on whatever shared memory
+// and TMEM hold, i.e. the tensor-core rate this kernel could reach if nothing else cost time.
+template <bool MMA_ONLY>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
                        const __grid_constant__ CUtensorMap tmap_y, const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
-                       int64_t ldy, int M, int N, int K, StatusWord *status, int probe, int group_m)
+                       int64_t ldy, int M, int N, int K, StatusWord *status, int group_m)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -215,7 +219,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const int num_ks = (katoms + kKbPerStage - 1) / kKbPerStage;
     const int pair = blockIdx.x >> 1;
     const int npairs = gridDim.x >> 1;
-    const int gm = (probe >> 8) > 0 ? (probe >> 8) : group_m;
+    const int gm = group_m;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -240,7 +244,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         mbar_expect_tx(sf_full_bar(stage), 2u * (SFA_BYTES + SFB_BYTES));
                         mbar_expect_tx(full_bar(stage), 2u * (A_BYTES + B_BYTES));
                     }
-                    if (!(probe & 2)) {
+                    if (!MMA_ONLY) {
                         tma2_load_2d(sSFA, &tmap_sfa, 0, rowblk * katoms + ks * kKbPerStage, leader_sf_full);
                         tma2_load_2d(sSFB, &tmap_sfw, 0, (2 * nb) * katoms + ks * kKbPerStage, leader_sf_full);
                         tma2_load_2d(sSFB + kKbPerStage * 512, &tmap_sfw, 0, (2 * nb + 1) * katoms + ks * kKbPerStage,
@@ -277,7 +281,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     const uint32_t b_lo = a_lo + (A_BYTES >> 4);
                     const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
                     const uint32_t t_sfb = t_sfa + 16u;
-                    if (!(probe & 1)) {
+                    {
                         if (ks == 0) mma2_nvf4<false>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
                         else mma2_nvf4<true>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
 #pragma unroll
@@ -315,7 +319,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         const uint32_t sfb_lo = sfa_lo + (SFA_BYTES >> 4);
                         const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
                         const uint32_t t_sfb = t_sfa + 16u;
-                        if (!(probe & 4)) {
+                        if (!MMA_ONLY) {
 #pragma unroll
                             for (int kb = 0; kb < kKbPerStage; ++kb) {
                                 if (kb < nkb) {
@@ -362,7 +366,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             // a TMA store, so that global memory sees full 128-byte lines instead of 16-byte pieces
             const int row0 = (mb * 2 + (int)rank) * BM + wq * 32;
             const int col0 = nb * BN + half * 128;
-            if (!(probe & 32)) {
+            if (!MMA_ONLY) {
                 const uint32_t stg = smem_base + STG_OFF + (uint32_t)ew * STG_WARP_BYTES;
                 const uint32_t my_row = stg + (uint32_t)lane * 128u;
                 const uint32_t sw = (uint32_t)(lane & 7);
@@ -452,12 +456,16 @@ bool make_y_tmap(EncodeTiledFn enc, CUtensorMap *tm, void *ptr, int64_t M, int64
 cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStream_t stream)
 {
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(encode_fn);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const int64_t katoms = a.K / 64;
     CUtensorMap tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y;
@@ -466,8 +474,6 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     if (!make_sf_tmap(enc, &tmap_sfa, a.a_sf, ((a.M + 127) / 128) * katoms)) return cudaErrorInvalidValue;
     if (!make_sf_tmap(enc, &tmap_sfw, a.w_sf, ((a.N + 255) / 256) * 2 * katoms)) return cudaErrorInvalidValue;
     if (!make_y_tmap(enc, &tmap_y, a.Y, a.M, a.N, a.ldy)) return cudaErrorInvalidValue;
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
     int pairs = sms / 2;
@@ -486,9 +492,13 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+    if (a.mma_only)
+        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<true>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+                                  a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M,
+                                  (int)a.N, (int)a.K, a.status, group_m);
+    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                               a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M, (int)a.N,
-                              (int)a.K, a.status, a.probe, group_m);
+                              (int)a.K, a.status, group_m);
 }
 
 }  // namespace dq

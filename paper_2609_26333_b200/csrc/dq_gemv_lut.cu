@@ -450,10 +450,9 @@ template <int BITS, int MAXT, int MINB>
 cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int threads, const LutPlan &L, uint32_t smem,
                        cudaStream_t stream)
 {
-    static bool attr_set[64] = {};
+    static bool attr_set[kMaxDevices] = {};
     int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);

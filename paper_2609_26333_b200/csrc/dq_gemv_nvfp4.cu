@@ -287,12 +287,14 @@ template <int BT, int MAXT>
 cudaError_t launch_one(const GemvNvArgs &a, const uint8_t *table, int b0, int grid, int threads, int W, int G,
                        cudaStream_t stream)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};
+    int attr_dev = 0;
+    if (cudaGetDevice(&attr_dev) != cudaSuccess || attr_dev < 0 || attr_dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[attr_dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemv_nvfp4_kernel<BT, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kDynSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[attr_dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

@@ -531,6 +531,38 @@ cudaError_t launch_import_lut(int bits, const uint32_t *planes_in, const uint8_t
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------ measurement kernel
+
+// Read-only streaming sum with 128-bit loads: the practical ceiling of a kernel that only reads (the decode
+// kernels' roofline is quoted against the copy bandwidth; this number shows what a pure reader reaches).
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4 *__restrict__ src, size_t n16, unsigned long long *out)
+{
+    uint32_t acc = 0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n16; i += 4 * stride) {          // four independent loads in flight per thread
+        const uint4 a = __ldg(src + i), b = __ldg(src + i + stride), c = __ldg(src + i + 2 * stride), d = __ldg(src + i + 3 * stride);
+        acc += (a.x ^ a.y ^ a.z ^ a.w) + (b.x ^ b.y ^ b.z ^ b.w) + (c.x ^ c.y ^ c.z ^ c.w) + (d.x ^ d.y ^ d.z ^ d.w);
+    }
+    for (; i < n16; i += stride) {
+        const uint4 a = __ldg(src + i);
+        acc += a.x ^ a.y ^ a.z ^ a.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0 && acc == 0x9E3779B9u) atomicAdd(out, 1ull);     // keeps the loads alive; almost never taken
+}
+
+cudaError_t launch_stream_read(const void *src_dev, size_t bytes, void *out_dev, cudaStream_t stream)
+{
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    stream_read_kernel<<<sms * 4, 512, 0, stream>>>(reinterpret_cast<const uint4 *>(src_dev), bytes / 16,
+                                                    reinterpret_cast<unsigned long long *>(out_dev));
+    return cudaGetLastError();
+}
+
 // --------------------------------------------------- activation quantiser
 
 // eight floats -> four bytes of E2M1 codes (element 0 in the low nibble of byte 0)

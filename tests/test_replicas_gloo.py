@@ -51,3 +51,24 @@ def test_single_process_is_identity():
 
     assert replicas.max_over_ranks([3.0, 1.5]) == [3.0, 1.5]
     assert replicas.whole_job_rate(2.0, 1, 1000.0) == 2.0
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_several_gpus():
+    """`bench.py --gpus 2` outside a launcher re-executes itself as two ranks; the CPU arm prints one line (rank 0)
+    that says n_gpus 2, the other rank exits without work."""
+    import json
+    import subprocess
+
+    sys.path.insert(0, ROOT)
+    from paper_2609_26333_b200 import replicas
+
+    cmd = replicas.spawn_command(3, ["x.py", "--a", 1], master_port=1234)
+    assert cmd[1:] == ["-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=3", "--master-addr", "127.0.0.1",
+                       "--master-port", "1234", "x.py", "--a", "1"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                          "--warmup", "0", "--workload", "c1_tiny", "--ref-rows", "16"], capture_output=True, text=True,
+                         env=env, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
