@@ -78,6 +78,12 @@ def lib() -> ctypes.CDLL:
         L.dqo_quant_lut2.argtypes = [f32p, i64, i64, i64, c.c_float, u16p, u32p, u8p]
         L.dqo_dequant_lut2.restype = None
         L.dqo_dequant_lut2.argtypes = [u32p, u8p, i64, i64, c.c_float, u16p, f64p]
+        L.dqo_rmsnorm_bf16.restype = None
+        L.dqo_rmsnorm_bf16.argtypes = [f32p, i64, i64, i64, f32p, c.c_float, f32p]
+        L.dqo_silu_f32.restype = c.c_float
+        L.dqo_silu_f32.argtypes = [c.c_float]
+        L.dqo_silu_mul_bf16.restype = None
+        L.dqo_silu_mul_bf16.argtypes = [f32p, i64, i64, i64, f32p]
         L.dqo_autocast_lut3_to_nvfp4.restype = None
         L.dqo_autocast_lut3_to_nvfp4.argtypes = [u32p, u8p, i64, i64, u16p, u8p, u8p]
         L.dqo_dequant_nvfp4.restype = None
@@ -212,6 +218,44 @@ def quant_lut2(x, s: float, codebook_f16=None):
     lib().dqo_quant_lut2(_p(x, ctypes.c_float), rows, K, K, np.float32(s), _p(cb, ctypes.c_uint16),
                          _p(planes, ctypes.c_uint32), _p(scales, ctypes.c_uint8))
     return planes, scales
+
+
+def rmsnorm_bf16(x, gamma, eps: float) -> np.ndarray:
+    """RMSNorm of a (rows, K) fp32 matrix (bf16 values) with weight gamma, result rounded to bf16 (App. C.1 fused
+    activation processing; fp32 arithmetic as fixed in dq_oracle.c).  Returns fp32 holding bf16 values."""
+    x = _f32_2d(x)
+    rows, K = x.shape
+    assert K % BLOCK == 0
+    g = np.ascontiguousarray(gamma, dtype=np.float32)
+    assert g.shape == (K,)
+    h = np.zeros((rows, K), dtype=np.float32)
+    lib().dqo_rmsnorm_bf16(_p(x, ctypes.c_float), rows, K, K, _p(g, ctypes.c_float), np.float32(eps), _p(h, ctypes.c_float))
+    return h
+
+
+def silu_f32(g: float) -> float:
+    return float(lib().dqo_silu_f32(np.float32(g)))
+
+
+def silu_mul_bf16(gate_up) -> np.ndarray:
+    """bf16( SiLU(gate) * up ) for a (rows, 2F) fp32 matrix [gate | up] (App. C.1 fused activation processing)."""
+    gu = _f32_2d(gate_up)
+    rows, F2 = gu.shape
+    assert F2 % 2 == 0
+    F = F2 // 2
+    h = np.zeros((rows, F), dtype=np.float32)
+    lib().dqo_silu_mul_bf16(_p(gu, ctypes.c_float), rows, F, F2, _p(h, ctypes.c_float))
+    return h
+
+
+def rmsnorm_quant_nvfp4(x, gamma, eps: float, act_scale: float):
+    """Fused RMSNorm + NVFP4 activation quantiser: the quantiser applied to the bf16-rounded norm output."""
+    return quant_nvfp4(rmsnorm_bf16(x, gamma, eps), act_scale)
+
+
+def silu_mul_quant_nvfp4(gate_up, act_scale: float):
+    """Fused SiLU(gate)*up + NVFP4 activation quantiser."""
+    return quant_nvfp4(silu_mul_bf16(gate_up), act_scale)
 
 
 def autocast_lut3_to_nvfp4(planes, lut_scales, codebook_f16=None):

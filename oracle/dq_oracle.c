@@ -384,6 +384,85 @@ void dqo_autocast_lut3_to_nvfp4(const uint32_t *planes, const uint8_t *lut_scale
     }
 }
 
+/* ------------------------------------------- activation processing + quantiser */
+
+/* The paper's prefill stack fuses activation processing with the NVFP4 activation quantiser (App. C.1
+ * "we fuse compatible projections and activation processing"; the per-component latency table counts the
+ * quantiser inside "norms").  It gives no arithmetic for the fused operators.  Reading used here: the fused
+ * operator produces exactly what the two unfused steps would -- the processed activation rounded to bf16
+ * (the dtype activations travel in), then dqo_quant_nvfp4 with the static input scale -- with the fp32
+ * arithmetic of the processing step fixed as follows so that it can be reproduced bit for bit:
+ *
+ * RMSNorm:  ss  = sum_k x_k^2      in fp32: x_k^2 summed in order inside each 16-element block, the block sums
+ *                                  combined 32 blocks at a time by a balanced binary tree (neighbours first), the
+ *                                  group sums added in increasing order
+ *           r   = 1 / sqrt(ss / K + eps)                      (fp32 divide, add, square root, reciprocal)
+ *           h_k = bf16( (x_k * r) * gamma_k )
+ * SiLU(gate) * up:  silu(g) = g / (1 + e),  e = 2^t,  t = clamp(g * (-log2 e), -126, 126), evaluated as
+ *           n = rint(t), f = fma(g, -L_hi, -n) then f = fma(g, -L_lo, f) with log2 e = L_hi + L_lo (so that the
+ *           reduction keeps full precision for large |g|), p = degree-7 polynomial in f with the Taylor
+ *           coefficients of 2^f (fused multiply-adds, highest degree first), e = p * 2^n;   h = bf16( silu(g) * u ).
+ * Outputs are fp32 arrays holding bf16 values. */
+static float dqo_round_to_bf16(float v) { return dqo_bf16_decode(dqo_bf16_encode(v)); }
+
+void dqo_rmsnorm_bf16(const float *x, int64_t rows, int64_t K, int64_t ld, const float *gamma, float eps, float *h)
+{
+    const int64_t nb = K / DQO_BLOCK;
+    const int64_t ngroups = (nb + 31) / 32;
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const float *xr = x + r * ld;
+        float total = 0.0f;
+        for (int64_t g = 0; g < ngroups; ++g) {
+            float v[32];
+            for (int i = 0; i < 32; ++i) {
+                int64_t b = g * 32 + i;
+                float bs = 0.0f;
+                if (b < nb)
+                    for (int k = 0; k < DQO_BLOCK; ++k) { float sq = xr[b * DQO_BLOCK + k] * xr[b * DQO_BLOCK + k]; bs = bs + sq; }
+                v[i] = bs;
+            }
+            for (int step = 1; step < 32; step *= 2)          /* neighbours first */
+                for (int i = 0; i < 32; i += 2 * step) v[i] = v[i] + v[i + step];
+            total = total + v[0];
+        }
+        float mean = total / (float)K;
+        float rr = 1.0f / sqrtf(mean + eps);
+        for (int64_t k = 0; k < K; ++k) {
+            float t = xr[k] * rr;
+            h[r * K + k] = dqo_round_to_bf16(t * gamma[k]);
+        }
+    }
+}
+
+float dqo_silu_f32(float g)
+{
+    static const float C[8] = { 1.0f, 0.6931471805599453f, 0.2402265069591007f, 0.05550410866482158f,
+                                0.009618129107628477f, 0.0013333558146428443f, 0.00015403530393381608f,
+                                1.5252733804059841e-05f };
+    const float L_HI = 1.4426950216293335f, L_LO = 1.925963033500256e-08f;      /* log2(e) = L_HI + L_LO */
+    float t = g * -L_HI;
+    float n = nearbyintf(fminf(fmaxf(t, -126.0f), 126.0f));
+    float f = fmaf(g, -L_HI, -n);
+    f = fmaf(g, -L_LO, f);
+    f = fminf(fmaxf(f, -1.0f), 1.0f);                 /* only clamped arguments (|g| > 87) leave [-0.5, 0.5] */
+    float p = C[7];
+    for (int i = 6; i >= 0; --i) p = fmaf(p, f, C[i]);
+    float e = ldexpf(p, (int)n);
+    return g / (1.0f + e);
+}
+
+/* gate_up: rows x 2F (gate in columns [0, F), up in [F, 2F): the output of a fused gate/up projection) */
+void dqo_silu_mul_bf16(const float *gate_up, int64_t rows, int64_t F, int64_t ld, float *h)
+{
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < F; ++k) {
+            float sv = dqo_silu_f32(gate_up[r * ld + k]);
+            h[r * F + k] = dqo_round_to_bf16(sv * gate_up[r * ld + F + k]);
+        }
+}
+
 /* ------------------------------------------------------------ dequantise */
 
 /* x^ = s * d_b * level, evaluated in double from exactly representable factors. */
