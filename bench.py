@@ -485,6 +485,33 @@ def main():
         if st != 0:
             raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the measurement hooks")
 
+    # ---- the activation stage fused with the operator in front of it (outside the timed region): the stand-alone
+    #      quantiser against RMSNorm + quantiser in one kernel (K wide) and, for the stage in front of a down
+    #      projection of this width, SiLU(gate)*up + quantiser on a [gate | up] matrix of 2K columns
+    fused = None
+    if not args.no_b2b:
+        def timed(fn, n=10):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            b0.record()
+            for _ in range(n):
+                fn()
+            b1.record()
+            torch.cuda.synchronize()
+            return b0.elapsed_time(b1) / n
+        gamma = torch.ones(K, dtype=torch.bfloat16, device=dev)
+        Mf = min(M, 4096)
+        GU = torch.randn(Mf, 2 * K, generator=torch.Generator(device=dev).manual_seed(5), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        q_only = timed(lambda: dq.prefill_quantize(ws[0], A, sa, workspace))
+        n_q = timed(lambda: dq.prefill_rmsnorm_quantize(ws[0], A, gamma, 1e-6, sa, workspace))
+        s_q = timed(lambda: dq.prefill_silu_mul_quantize(ws[0], GU, sa, workspace))
+        fused = {"quantize_ms": q_only, "rmsnorm_quantize_ms": n_q, "rmsnorm_quantize_gbs": 2.5625 * M * K / (n_q * 1e-3) / 1e9,
+                 "silu_mul_quantize_ms": s_q, "silu_mul_rows": Mf, "silu_mul_quantize_gbs": 4.5625 * Mf * K / (s_q * 1e-3) / 1e9,
+                 "note": "unfused, the bf16 intermediate costs a write and a read of 2 bytes per element (4 of the 6.56 "
+                         "bytes per element of norm + quantiser) that the fused kernels do not make"}
+        del GU
+
     # ---- end to end: pinned host buffers, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -595,6 +622,8 @@ def main():
                                     "frac": l2_bytes / (d_l2_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                                     "ms": d_l2_ms, "timing": "back-to-back launches",
                                     "peak_source": f"{peaks['source']} copy bandwidth"}
+    if fused:
+        line["fused_activation_stage"] = fused
     if e2e:
         line["e2e"] = {"value": world * flops / (e2e_p_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": int(2 * M * K + 2 * B * K), "d2h_bytes_per_step": int(2 * M * N + 2 * B * N),

@@ -142,6 +142,27 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
                     const void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * The activation stage of the prefill linear fused with the operator in front of it, so that the normalised or gated
+ * activation never travels through HBM (App. C.1: the paper's prefill stack fuses activation processing with the
+ * activation quantiser; its per-component latency table counts the quantiser inside "norms").  Each call replaces
+ * dq_prefill_quantize and is followed by dq_prefill_gemm with the same M, workspace and act_global_scale.
+ *   dq_prefill_rmsnorm_quantize:  A = bf16( X * r * gamma ),  r = 1 / sqrt(mean_k(X^2) + eps) per row,
+ *       X_dev: M x K bf16 (row stride ldx), gamma_dev: K bf16 (16-byte aligned), eps >= 0; K <= 131072.
+ *   dq_prefill_silu_mul_quantize: A = bf16( SiLU(G) * U ),  SiLU(g) = g / (1 + exp(-g)),
+ *       GU_dev: M x 2K bf16 (row stride ldgu >= 2K), G in columns [0, K), U in [K, 2K): the output of a fused
+ *       gate/up projection feeding the down projection `w`.
+ * A is what the two unfused steps would produce (the operator's result rounded to bf16); it is quantised exactly as
+ * dq_prefill_quantize quantises (App. A.3 "NVFP4", static input scale).  The fp32 arithmetic of r and of exp is
+ * fixed (stated at the top of csrc/dq_fused_quant.cu), so codes and scales are reproducible bit for bit.
+ */
+int dq_prefill_rmsnorm_quantize(const dq_weights *w, const void *X_dev, int64_t M, int64_t ldx,
+                                const void *gamma_dev, float eps, float act_global_scale,
+                                void *workspace_dev, size_t workspace_bytes, void *stream);
+int dq_prefill_silu_mul_quantize(const dq_weights *w, const void *GU_dev, int64_t M, int64_t ldgu,
+                                 float act_global_scale, void *workspace_dev, size_t workspace_bytes,
+                                 void *stream);
+
+/*
  * dq_prefill_linear without a caller-provided workspace.  (The paper has no counterpart: this
  * entry point exists for integration, not for the method.)
  * It is meant for callers that cannot allocate device memory where they call from -- an engine
@@ -265,6 +286,17 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
 int dq_quantize_activations(const void *A_dev, int64_t M, int64_t K, int64_t lda,
                             float act_global_scale, void *codes_dev, void *scales_dev,
                             void *stream);
+
+/*
+ * The fused quantisers of dq_prefill_rmsnorm_quantize / dq_prefill_silu_mul_quantize on their own, writing canonical
+ * layout (codes uint8[M][K/2], scales uint8[M][K/16]; K = F for the gated form).  Arguments as there.
+ */
+int dq_rmsnorm_quantize_activations(const void *X_dev, int64_t M, int64_t K, int64_t ldx,
+                                    const void *gamma_dev, float eps, float act_global_scale,
+                                    void *codes_dev, void *scales_dev, void *stream);
+int dq_silu_mul_quantize_activations(const void *GU_dev, int64_t M, int64_t F, int64_t ldgu,
+                                     float act_global_scale, void *codes_dev, void *scales_dev,
+                                     void *stream);
 
 /*
  * Reads the library's device status word for the current device (synchronises

@@ -22,7 +22,9 @@ SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
            "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear",
-           "dq_bench_gemm_mma_only", "dq_bench_stream_read", "dq_export_canonical", "dq_import_canonical",
+           "dq_bench_gemm_mma_only", "dq_bench_stream_read",
+           "dq_prefill_rmsnorm_quantize", "dq_prefill_silu_mul_quantize", "dq_rmsnorm_quantize_activations",
+           "dq_silu_mul_quantize_activations", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
            "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
@@ -81,6 +83,14 @@ def lib() -> C.CDLL:
         L.dq_test_decode_linear.restype = C.c_int
         L.dq_test_decode_linear.argtypes = [vp, C.c_uint, C.c_int, C.c_int, C.c_int, C.c_int, C.c_longlong, vp, i64, i64,
                                             vp, i64, vp]
+        L.dq_prefill_rmsnorm_quantize.restype = C.c_int
+        L.dq_prefill_rmsnorm_quantize.argtypes = [vp, vp, i64, i64, vp, C.c_float, C.c_float, vp, sz, vp]
+        L.dq_prefill_silu_mul_quantize.restype = C.c_int
+        L.dq_prefill_silu_mul_quantize.argtypes = [vp, vp, i64, i64, C.c_float, vp, sz, vp]
+        L.dq_rmsnorm_quantize_activations.restype = C.c_int
+        L.dq_rmsnorm_quantize_activations.argtypes = [vp, i64, i64, i64, vp, C.c_float, C.c_float, vp, vp, vp]
+        L.dq_silu_mul_quantize_activations.restype = C.c_int
+        L.dq_silu_mul_quantize_activations.argtypes = [vp, i64, i64, i64, C.c_float, vp, vp, vp]
         L.dq_bench_gemm_mma_only.restype = C.c_int
         L.dq_bench_gemm_mma_only.argtypes = [vp, i64, vp, i64, vp, sz, vp]
         L.dq_bench_stream_read.restype = C.c_int
@@ -243,6 +253,46 @@ def prefill_quantize(w: DQWeights, A: torch.Tensor, act_global_scale: float, wor
     _check(lib().dq_prefill_quantize(w.handle, A.data_ptr(), A.shape[0], A.stride(0), float(act_global_scale),
                                      workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
            "dq_prefill_quantize")
+
+
+def prefill_rmsnorm_quantize(w: DQWeights, X: torch.Tensor, gamma: torch.Tensor, eps: float, act_global_scale: float,
+                             workspace: torch.Tensor, stream=None):
+    """dq_prefill_rmsnorm_quantize: RMSNorm fused with stage 1 of the prefill linear."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.stride(1) == 1 and X.shape[1] == w.K
+    assert gamma.is_cuda and gamma.dtype == torch.bfloat16 and gamma.is_contiguous() and gamma.numel() == w.K
+    _check(lib().dq_prefill_rmsnorm_quantize(w.handle, X.data_ptr(), X.shape[0], X.stride(0), gamma.data_ptr(), float(eps),
+                                             float(act_global_scale), workspace.data_ptr(), workspace.numel(),
+                                             _stream_ptr(stream)), "dq_prefill_rmsnorm_quantize")
+
+
+def prefill_silu_mul_quantize(w: DQWeights, GU: torch.Tensor, act_global_scale: float, workspace: torch.Tensor, stream=None):
+    """dq_prefill_silu_mul_quantize: SiLU(gate) * up fused with stage 1 of the prefill linear (GU = [gate | up])."""
+    assert GU.is_cuda and GU.dtype == torch.bfloat16 and GU.stride(1) == 1 and GU.shape[1] == 2 * w.K
+    _check(lib().dq_prefill_silu_mul_quantize(w.handle, GU.data_ptr(), GU.shape[0], GU.stride(0), float(act_global_scale),
+                                              workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)),
+           "dq_prefill_silu_mul_quantize")
+
+
+def rmsnorm_quantize_activations(X: torch.Tensor, gamma: torch.Tensor, eps: float, act_global_scale: float, stream=None):
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    codes = torch.empty(M, K // 2, dtype=torch.uint8, device=X.device)
+    scales = torch.empty(M, K // 16, dtype=torch.uint8, device=X.device)
+    _check(lib().dq_rmsnorm_quantize_activations(X.data_ptr(), M, K, X.stride(0), gamma.data_ptr(), float(eps),
+                                                 float(act_global_scale), codes.data_ptr(), scales.data_ptr(),
+                                                 _stream_ptr(stream)), "dq_rmsnorm_quantize_activations")
+    return codes, scales
+
+
+def silu_mul_quantize_activations(GU: torch.Tensor, act_global_scale: float, stream=None):
+    assert GU.is_cuda and GU.dtype == torch.bfloat16 and GU.dim() == 2 and GU.stride(1) == 1 and GU.shape[1] % 2 == 0
+    M, F = GU.shape[0], GU.shape[1] // 2
+    codes = torch.empty(M, F // 2, dtype=torch.uint8, device=GU.device)
+    scales = torch.empty(M, F // 16, dtype=torch.uint8, device=GU.device)
+    _check(lib().dq_silu_mul_quantize_activations(GU.data_ptr(), M, F, GU.stride(0), float(act_global_scale),
+                                                  codes.data_ptr(), scales.data_ptr(), _stream_ptr(stream)),
+           "dq_silu_mul_quantize_activations")
+    return codes, scales
 
 
 def prefill_gemm(w: DQWeights, M: int, act_global_scale: float, out: torch.Tensor, workspace: torch.Tensor,

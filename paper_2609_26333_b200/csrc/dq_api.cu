@@ -323,6 +323,19 @@ static int prefill_checks(const dq_weights *w, int64_t M, float act_global_scale
     return DQ_OK;
 }
 
+// the part of the activation stage that does not depend on how the activations were produced: for a handle that stores
+// only LUT3, cast the weights to NVFP4 for this call (Sec. 2.3, same code map as the pack-time view); rows that pad the
+// scale layout to the GEMM tile must read as zero
+static int prefill_weight_view(const dq_weights *w, uint8_t *ws, const WsLayout &L, cudaStream_t s)
+{
+    if (has_nvfp4_view(w)) return DQ_OK;
+    if (w->N % dq::kSfRowPad != 0 && cudaMemsetAsync(ws + L.w_sf, 0, L.w_sf_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_autocast(reinterpret_cast<const dq::PackedHeader *>(w->base), w->base + w->layout.lut_off, w->N, w->K,
+                            ws + L.w_codes, ws + L.w_sf, s) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
 int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64_t lda, float act_global_scale,
                         void *workspace_dev, size_t workspace_bytes, void *stream)
 {
@@ -337,16 +350,44 @@ int dq_prefill_quantize(const dq_weights *w, const void *A_dev, int64_t M, int64
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (dq::launch_quant_act(A_dev, M, w->K, lda, act_global_scale, ws, ws + L.a_sf, 1, s) != cudaSuccess)
         return DQ_ERR_CUDA;
-    if (!has_nvfp4_view(w)) {
-        // the stored matrix is LUT3 only: cast it to NVFP4 for this call (Sec. 2.3, same code map as the
-        // pack-time view); rows that pad the scale layout to the GEMM tile must read as zero
-        if (w->N % dq::kSfRowPad != 0 && cudaMemsetAsync(ws + L.w_sf, 0, L.w_sf_bytes, s) != cudaSuccess)
-            return DQ_ERR_CUDA;
-        if (dq::launch_autocast(reinterpret_cast<const dq::PackedHeader *>(w->base), w->base + w->layout.lut_off, w->N,
-                                w->K, ws + L.w_codes, ws + L.w_sf, s) != cudaSuccess)
-            return DQ_ERR_CUDA;
-    }
-    return DQ_OK;
+    return prefill_weight_view(w, ws, L, s);
+}
+
+int dq_prefill_rmsnorm_quantize(const dq_weights *w, const void *X_dev, int64_t M, int64_t ldx, const void *gamma_dev,
+                                float eps, float act_global_scale, void *workspace_dev, size_t workspace_bytes,
+                                void *stream)
+{
+    if (!X_dev || !gamma_dev) return DQ_ERR_INVALID_ARG;
+    if (!(eps >= 0.0f) || !std::isfinite(eps)) return DQ_ERR_INVALID_ARG;
+    int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (w->K > 131072) return DQ_ERR_SHAPE;
+    if (ldx < w->K || ldx % 8 != 0 || !aligned(X_dev, 16) || !aligned(gamma_dev, 16)) return DQ_ERR_ALIGN;
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
+    const WsLayout L = ws_layout(w, M);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (dq::launch_rmsnorm_quant(X_dev, M, w->K, ldx, gamma_dev, eps, act_global_scale, ws, ws + L.a_sf, 1, s) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return prefill_weight_view(w, ws, L, s);
+}
+
+int dq_prefill_silu_mul_quantize(const dq_weights *w, const void *GU_dev, int64_t M, int64_t ldgu, float act_global_scale,
+                                 void *workspace_dev, size_t workspace_bytes, void *stream)
+{
+    if (!GU_dev) return DQ_ERR_INVALID_ARG;
+    int st = prefill_checks(w, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (ldgu < 2 * w->K || ldgu % 8 != 0 || !aligned(GU_dev, 16)) return DQ_ERR_ALIGN;
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace_dev);
+    const WsLayout L = ws_layout(w, M);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (dq::launch_silu_mul_quant(GU_dev, M, w->K, ldgu, act_global_scale, ws, ws + L.a_sf, 1, s) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return prefill_weight_view(w, ws, L, s);
 }
 
 static int prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void *Y_dev, int64_t ldy,
@@ -550,6 +591,42 @@ int dq_quantize_activations(const void *A_dev, int64_t M, int64_t K, int64_t lda
     if (dq::launch_quant_act(A_dev, M, K, lda, act_global_scale, reinterpret_cast<uint8_t *>(codes_dev),
                              reinterpret_cast<uint8_t *>(scales_dev), 0,
                              reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_rmsnorm_quantize_activations(const void *X_dev, int64_t M, int64_t K, int64_t ldx, const void *gamma_dev, float eps,
+                                    float act_global_scale, void *codes_dev, void *scales_dev, void *stream)
+{
+    if (!X_dev || !gamma_dev || !codes_dev || !scales_dev) return DQ_ERR_INVALID_ARG;
+    if (M < 1 || K < 1 || K % 128 != 0 || K > 131072) return DQ_ERR_SHAPE;
+    if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
+    if (!(eps >= 0.0f) || !std::isfinite(eps)) return DQ_ERR_INVALID_ARG;
+    if (ldx < K || ldx % 8 != 0 || !aligned(X_dev, 16) || !aligned(gamma_dev, 16) || !aligned(codes_dev, 16) ||
+        !aligned(scales_dev, 4))
+        return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    if (dq::launch_rmsnorm_quant(X_dev, M, K, ldx, gamma_dev, eps, act_global_scale, reinterpret_cast<uint8_t *>(codes_dev),
+                                 reinterpret_cast<uint8_t *>(scales_dev), 0, reinterpret_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
+        return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_silu_mul_quantize_activations(const void *GU_dev, int64_t M, int64_t F, int64_t ldgu, float act_global_scale,
+                                     void *codes_dev, void *scales_dev, void *stream)
+{
+    if (!GU_dev || !codes_dev || !scales_dev) return DQ_ERR_INVALID_ARG;
+    if (M < 1 || F < 1 || F % 128 != 0) return DQ_ERR_SHAPE;
+    if (!(act_global_scale > 0.0f) || !std::isfinite(act_global_scale)) return DQ_ERR_INVALID_ARG;
+    if (ldgu < 2 * F || ldgu % 8 != 0 || !aligned(GU_dev, 16) || !aligned(codes_dev, 16) || !aligned(scales_dev, 4))
+        return DQ_ERR_ALIGN;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    if (dq::launch_silu_mul_quant(GU_dev, M, F, ldgu, act_global_scale, reinterpret_cast<uint8_t *>(codes_dev),
+                                  reinterpret_cast<uint8_t *>(scales_dev), 0, reinterpret_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
         return DQ_ERR_CUDA;
     return DQ_OK;
 }

@@ -189,6 +189,12 @@ cudaError_t launch_import_lut(int bits, const uint32_t *planes_in, const uint8_t
 cudaError_t launch_quant_act(const void *A_bf16, int64_t M, int64_t K, int64_t lda, float act_scale, uint8_t *codes,
                              uint8_t *sf, int swizzled, cudaStream_t stream);
 
+// fused activation processing + quantiser (dq_fused_quant.cu); outputs as launch_quant_act
+cudaError_t launch_rmsnorm_quant(const void *X_bf16, int64_t M, int64_t K, int64_t ldx, const void *gamma_bf16, float eps,
+                                 float act_scale, uint8_t *codes, uint8_t *sf, int swizzled, cudaStream_t stream);
+cudaError_t launch_silu_mul_quant(const void *GU_bf16, int64_t M, int64_t F, int64_t ldgu, float act_scale, uint8_t *codes,
+                                  uint8_t *sf, int swizzled, cudaStream_t stream);
+
 struct GemmArgs {
     const uint8_t *a_codes;  const uint8_t *a_sf;      // activations: [M][K/2], MMA scale layout
     const uint8_t *w_codes;  const uint8_t *w_sf;      // weights:     [N][K/2], MMA scale layout
