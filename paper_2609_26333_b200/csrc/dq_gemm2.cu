@@ -31,28 +31,41 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128;                       // rows per CTA (pair tile: 256)
-constexpr int BN = 256;
-constexpr int kStages = 5;
-constexpr int kKbPerStage = 4;                // 64-element MMA k-steps per 256-element stage
-constexpr uint32_t A_BYTES = BM * 128;        // 16 KiB: 128 rows x 128 B of packed FP4
-constexpr uint32_t B_BYTES = (BN / 2) * 128;  // 16 KiB: this CTA's half of the W tile
-constexpr uint32_t SFA_BYTES = kKbPerStage * 512;
-constexpr uint32_t SFB_BYTES = 2 * kKbPerStage * 512;
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 38 KiB
-constexpr uint32_t STG_WARP_BYTES = 32 * 128;                                  // 32 rows x 64 bf16, one TMA-store box
-constexpr uint32_t STG_OFF = kStages * STAGE_BYTES;                           // epilogue staging, 1024-byte aligned
-constexpr uint32_t BAR_OFF = STG_OFF + 8 * STG_WARP_BYTES;
-constexpr uint32_t SMEM_BYTES = BAR_OFF + 1024 + 256;
-constexpr int kEpiWarps = 8;
-constexpr int kThreads = 128 + 32 * kEpiWarps;
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemSfBase = 256;
-constexpr uint32_t kTmemSfBufCols = 48;      // 16 (A) + 32 (B) columns per stage
-static_assert(kTmemSfBase + kStages * kTmemSfBufCols <= kTmemCols, "scale buffers must fit in TMEM");
-static_assert(STAGE_BYTES % 1024 == 0, "stages must stay 1024-byte aligned");
 
-// dense, A/B = E2M1, K-major, UE4M3 scales, N = 256, M = 256 across the pair
-constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+// Tile configuration: one 256 x 256 pair tile per step, one CTA per SM, the whole TMEM (256 accumulator columns +
+// 5 scale buffers of 48).  (A 256 x 128 configuration with two CTAs of different pairs per SM, meant to hide the
+// accumulator hand-off behind the other pair's MMAs, was measured 20 % slower on 8192 x 5120 x 17408 and is not
+// kept.)
+template <int BN_, int STAGES_, int EPI_WARPS_, int MIN_CTAS_>
+struct Cfg {
+    static constexpr int BN = BN_;
+    static constexpr int kStages = STAGES_;
+    static constexpr int kEpiWarps = EPI_WARPS_;
+    static constexpr int kMinCtas = MIN_CTAS_;
+    static constexpr int kKbPerStage = 4;                 // 64-element MMA k-steps per 256-element stage
+    static constexpr int kSfbAtoms = BN / 128;            // 128-row scale atoms of the W tile
+    static constexpr uint32_t A_BYTES = BM * 128;         // 16 KiB: 128 rows x 128 B of packed FP4
+    static constexpr uint32_t B_BYTES = (BN / 2) * 128;   // this CTA's half of the W tile
+    static constexpr uint32_t SFA_BYTES = kKbPerStage * 512;
+    static constexpr uint32_t SFB_BYTES = kSfbAtoms * kKbPerStage * 512;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+    static constexpr uint32_t STG_WARP_BYTES = 32 * 128;                          // 32 rows x 64 bf16, one TMA-store box
+    static constexpr uint32_t STG_OFF = kStages * STAGE_BYTES;                    // epilogue staging, 1024-byte aligned
+    static constexpr uint32_t BAR_OFF = STG_OFF + kEpiWarps * STG_WARP_BYTES;
+    static constexpr uint32_t SMEM_BYTES = BAR_OFF + 1024 + 256;
+    static constexpr int kThreads = 128 + 32 * kEpiWarps;
+    static constexpr uint32_t kTmemSfBase = BN;                                   // accumulator: BN fp32 columns
+    static constexpr uint32_t kTmemSfACols = 4 * kKbPerStage;
+    static constexpr uint32_t kTmemSfBufCols = kTmemSfACols + 4 * kKbPerStage * kSfbAtoms;
+    static constexpr uint32_t kTmemCols = (BN + kStages * kTmemSfBufCols) <= 256 ? 256 : 512;
+    static_assert(kTmemSfBase + kStages * kTmemSfBufCols <= kTmemCols, "scale buffers must fit in TMEM");
+    static_assert(STAGE_BYTES % 1024 == 0, "stages must stay 1024-byte aligned");
+    static_assert(kEpiWarps == 4 * (BN / 128), "four epilogue warps (one per TMEM lane quarter) per 128 columns");
+    // dense, A/B = E2M1, K-major, UE4M3 scales, N = BN, M = 256 across the pair
+    static constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+};
+using WideCfg = Cfg<256, 5, 8, 1>;
+
 constexpr uint32_t kDescHiSw128 = 64u | (1u << 14) | (2u << 29);   // SBO 1024 B, version 1, 128B swizzle
 constexpr uint32_t kDescHiSf = 8u | (1u << 14);                    // SBO 128 B, version 1, no swizzle
 
@@ -95,12 +108,12 @@ __device__ __forceinline__ void tmem2_cp_sf(uint32_t taddr, uint32_t lo, uint32_
 }
 template <bool ACC>
 __device__ __forceinline__ void mma2_nvf4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t sfa,
-                                          uint32_t sfb)
+                                          uint32_t sfb, uint32_t idesc)
 {
     asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
                  "setp.ne.b32 p, %7, 0;\n\t"
                  "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], da, db, %4, [%5], [%6], p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(kInstrDesc), "r"(sfa), "r"(sfb),
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(sfa), "r"(sfb),
                    "r"(ACC ? 1u : 0u) : "memory");
 }
 // TMA store of one staged box (shared -> global); out-of-range rows / columns are clipped by the hardware
@@ -163,13 +176,19 @@ __device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, in
 // MMA_ONLY (measurement): the same roles and barriers, but no operand or scale loads (the barriers are completed by
 // hand), no scale copies into TMEM and no stores: what is left is the MMA issue sequence on whatever shared memory
 // and TMEM hold, i.e. the tensor-core rate this kernel could reach if nothing else cost time.
-template <bool MMA_ONLY>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+template <bool MMA_ONLY, class C>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C::kThreads, C::kMinCtas)
 gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
                        const __grid_constant__ CUtensorMap tmap_y, const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
                        int64_t ldy, int M, int N, int K, StatusWord *status, int group_m)
 {
+    constexpr int BN = C::BN, kStages = C::kStages, kKbPerStage = C::kKbPerStage, kEpiWarps = C::kEpiWarps;
+    constexpr int kSfbAtoms = C::kSfbAtoms;
+    constexpr uint32_t A_BYTES = C::A_BYTES, B_BYTES = C::B_BYTES, SFA_BYTES = C::SFA_BYTES, SFB_BYTES = C::SFB_BYTES;
+    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES, STG_WARP_BYTES = C::STG_WARP_BYTES, STG_OFF = C::STG_OFF;
+    constexpr uint32_t BAR_OFF = C::BAR_OFF, kTmemCols = C::kTmemCols, kTmemSfBase = C::kTmemSfBase;
+    constexpr uint32_t kTmemSfBufCols = C::kTmemSfBufCols, kTmemSfACols = C::kTmemSfACols, kInstrDesc = C::kInstrDesc;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -246,9 +265,10 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     }
                     if (!MMA_ONLY) {
                         tma2_load_2d(sSFA, &tmap_sfa, 0, rowblk * katoms + ks * kKbPerStage, leader_sf_full);
-                        tma2_load_2d(sSFB, &tmap_sfw, 0, (2 * nb) * katoms + ks * kKbPerStage, leader_sf_full);
-                        tma2_load_2d(sSFB + kKbPerStage * 512, &tmap_sfw, 0, (2 * nb + 1) * katoms + ks * kKbPerStage,
-                                     leader_sf_full);
+#pragma unroll
+                        for (int at = 0; at < kSfbAtoms; ++at)
+                            tma2_load_2d(sSFB + (uint32_t)at * kKbPerStage * 512, &tmap_sfw, 0,
+                                         (kSfbAtoms * nb + at) * katoms + ks * kKbPerStage, leader_sf_full);
                         tma2_load_2d(sA, &tmap_a, ks * 128, rowblk * BM, leader_full);
                         tma2_load_2d(sB, &tmap_w, ks * 128, nb * BN + (int)rank * (BN / 2), leader_full);
                     } else if (rank == 0) {
@@ -280,15 +300,15 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     const uint32_t a_lo = a_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
                     const uint32_t b_lo = a_lo + (A_BYTES >> 4);
                     const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
-                    const uint32_t t_sfb = t_sfa + 16u;
+                    const uint32_t t_sfb = t_sfa + kTmemSfACols;
                     {
-                        if (ks == 0) mma2_nvf4<false>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
-                        else mma2_nvf4<true>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb);
+                        if (ks == 0) mma2_nvf4<false>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb, kInstrDesc);
+                        else mma2_nvf4<true>(tmem_base, a_lo, b_lo, kDescHiSw128, t_sfa, t_sfb, kInstrDesc);
 #pragma unroll
                         for (int kb = 1; kb < kKbPerStage; ++kb) {
                             if (kb < nkb)
                                 mma2_nvf4<true>(tmem_base, a_lo + 2u * kb, b_lo + 2u * kb, kDescHiSw128, t_sfa + 4u * kb,
-                                                t_sfb + 8u * kb);
+                                                t_sfb + 4u * kSfbAtoms * kb, kInstrDesc);
                         }
                     }
                     mma2_commit_pair(empty_bar(stage));     // stage (smem and TMEM scales) reusable in both CTAs
@@ -318,14 +338,16 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         const uint32_t sfa_lo = sf_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
                         const uint32_t sfb_lo = sfa_lo + (SFA_BYTES >> 4);
                         const uint32_t t_sfa = tmem_base + kTmemSfBase + (uint32_t)stage * kTmemSfBufCols;
-                        const uint32_t t_sfb = t_sfa + 16u;
+                        const uint32_t t_sfb = t_sfa + kTmemSfACols;
                         if (!MMA_ONLY) {
 #pragma unroll
                             for (int kb = 0; kb < kKbPerStage; ++kb) {
                                 if (kb < nkb) {
                                     tmem2_cp_sf(t_sfa + 4u * kb, sfa_lo + 32u * kb, kDescHiSf);
-                                    tmem2_cp_sf(t_sfb + 8u * kb, sfb_lo + 32u * kb, kDescHiSf);
-                                    tmem2_cp_sf(t_sfb + 8u * kb + 4u, sfb_lo + (kKbPerStage * 512u >> 4) + 32u * kb, kDescHiSf);
+#pragma unroll
+                                    for (int at = 0; at < kSfbAtoms; ++at)
+                                        tmem2_cp_sf(t_sfb + 4u * kSfbAtoms * kb + 4u * at,
+                                                    sfb_lo + (uint32_t)at * (kKbPerStage * 512u >> 4) + 32u * kb, kDescHiSf);
                                 }
                             }
                         }
@@ -350,46 +372,47 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             if (!mbar_wait2(tmem_full_bar, acc_phase, abort_flag, peer_abort)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(half * 128);
+            // bf16 rows go through a swizzled staging box (32 rows x 64 columns per warp) and leave with
+            // a TMA store, so that global memory sees full 128-byte lines instead of 16-byte pieces
+            const int row0 = (mb * 2 + (int)rank) * BM + wq * 32;
+            const int col0 = nb * BN + half * 128;
+            const uint32_t stg = smem_base + STG_OFF + (uint32_t)ew * STG_WARP_BYTES;
+            const uint32_t my_row = stg + (uint32_t)lane * 128u;
+            const uint32_t sw = (uint32_t)(lane & 7);
+            auto stage_box = [&](const uint32_t (&lo)[32], const uint32_t (&hi)[32], int box) {
+                if (MMA_ONLY) return;
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer free again
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t (&v)[32] = (c < 4) ? lo : hi;
+                    const int o = (c & 3) * 8;
+                    sts_v4(my_row + (((uint32_t)c ^ sw) << 4),
+                           pack_bf16x2(__uint_as_float(v[o + 0]) * alpha, __uint_as_float(v[o + 1]) * alpha),
+                           pack_bf16x2(__uint_as_float(v[o + 2]) * alpha, __uint_as_float(v[o + 3]) * alpha),
+                           pack_bf16x2(__uint_as_float(v[o + 4]) * alpha, __uint_as_float(v[o + 5]) * alpha),
+                           pack_bf16x2(__uint_as_float(v[o + 6]) * alpha, __uint_as_float(v[o + 7]) * alpha));
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && row0 < M && col0 + box * 64 < N) tma_store_2d(&tmap_y, stg, col0 + box * 64, row0);
+            };
+            auto release_tmem = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(leader_tmem_empty);
+            };
+            // the whole 128-column slice at once, TMEM handed back before converting and storing
             uint32_t v0[32], v1[32], v2[32], v3[32];
             tmem_ld32(taddr, v0);
             tmem_ld32(taddr + 32u, v1);
             tmem_ld32(taddr + 64u, v2);
             tmem_ld32(taddr + 96u, v3);
             tmem_ld_wait();
-            // the accumulator is in registers: hand TMEM back before converting and storing
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(leader_tmem_empty);
+            release_tmem();
+            stage_box(v0, v1, 0);
+            stage_box(v2, v3, 1);
             acc_phase ^= 1u;
-
-            // bf16 rows go through a swizzled staging box (32 rows x 64 columns per warp) and leave with
-            // a TMA store, so that global memory sees full 128-byte lines instead of 16-byte pieces
-            const int row0 = (mb * 2 + (int)rank) * BM + wq * 32;
-            const int col0 = nb * BN + half * 128;
-            if (!MMA_ONLY) {
-                const uint32_t stg = smem_base + STG_OFF + (uint32_t)ew * STG_WARP_BYTES;
-                const uint32_t my_row = stg + (uint32_t)lane * 128u;
-                const uint32_t sw = (uint32_t)(lane & 7);
-                auto stage_box = [&](const uint32_t (&lo)[32], const uint32_t (&hi)[32], int box) {
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer free again
-                    __syncwarp();
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint32_t (&v)[32] = (c < 4) ? lo : hi;
-                        const int o = (c & 3) * 8;
-                        sts_v4(my_row + (((uint32_t)c ^ sw) << 4),
-                               pack_bf16x2(__uint_as_float(v[o + 0]) * alpha, __uint_as_float(v[o + 1]) * alpha),
-                               pack_bf16x2(__uint_as_float(v[o + 2]) * alpha, __uint_as_float(v[o + 3]) * alpha),
-                               pack_bf16x2(__uint_as_float(v[o + 4]) * alpha, __uint_as_float(v[o + 5]) * alpha),
-                               pack_bf16x2(__uint_as_float(v[o + 6]) * alpha, __uint_as_float(v[o + 7]) * alpha));
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0 && row0 < M && col0 + box * 64 < N) tma_store_2d(&tmap_y, stg, col0 + box * 64, row0);
-                };
-                stage_box(v0, v1, 0);
-                stage_box(v2, v3, 1);
-            }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // all stores of this warp done
     }
@@ -432,7 +455,7 @@ bool make_sf_tmap(EncodeTiledFn enc, CUtensorMap *tm, const void *ptr, int64_t a
 {
     cuuint64_t gdim[2] = {128u, (cuuint64_t)atoms};
     cuuint64_t gstride[1] = {512u};
-    cuuint32_t box[2] = {128u, (cuuint32_t)kKbPerStage};
+    cuuint32_t box[2] = {128u, (cuuint32_t)4u};
     cuuint32_t estr[2] = {1u, 1u};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(ptr), gdim, gstride, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -451,22 +474,21 @@ bool make_y_tmap(EncodeTiledFn enc, CUtensorMap *tm, void *ptr, int64_t M, int64
            CUDA_SUCCESS;
 }
 
-}  // namespace
-
-cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStream_t stream)
+template <class C>
+static cudaError_t launch_pair_cfg(const GemmArgs &a, EncodeTiledFn enc, cudaStream_t stream)
 {
-    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(encode_fn);
     static bool attr_set[kMaxDevices] = {};
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false, C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             C::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<true, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
+    constexpr int BN = C::BN;
     const int64_t katoms = a.K / 64;
     CUtensorMap tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y;
     if (!make_codes_tmap2(enc, &tmap_a, a.a_codes, a.M, a.K, BM)) return cudaErrorInvalidValue;
@@ -476,7 +498,7 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     if (!make_y_tmap(enc, &tmap_y, a.Y, a.M, a.N, a.ldy)) return cudaErrorInvalidValue;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
-    int pairs = sms / 2;
+    int pairs = sms / 2 * C::kMinCtas;
     if (tiles < pairs) pairs = tiles;
     // Tile order: groups of group_m row tiles sweep all column tiles, so that the A rows of a group stay in L2
     // while each W tile is read once per group.  Largest power of two whose A codes + scales fit about 48 MB.
@@ -484,8 +506,8 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     while (group_m < 64 && (double)(2 * group_m) * 256.0 * (double)a.K * 0.5625 <= 48.0e6) group_m *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
-    cfg.blockDim = dim3((unsigned)kThreads);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.blockDim = dim3((unsigned)C::kThreads);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -493,12 +515,19 @@ cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStrea
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (a.mma_only)
-        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<true>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<true, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                                   a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M,
                                   (int)a.N, (int)a.K, a.status, group_m);
-    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                               a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M, (int)a.N,
                               (int)a.K, a.status, group_m);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &a, void *encode_fn, cudaStream_t stream)
+{
+    return launch_pair_cfg<WideCfg>(a, reinterpret_cast<EncodeTiledFn>(encode_fn), stream);
 }
 
 }  // namespace dq

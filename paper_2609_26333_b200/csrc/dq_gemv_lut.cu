@@ -484,7 +484,7 @@ static uint32_t plan_smem(int bits, int K, int P, int G, int S, int cols, LutPla
     L.P = P; L.G = G; L.S = S;
     L.bar_off = 1024;
     L.red_off = 2048;
-    const uint32_t red_bytes = (uint32_t)nwarps * kSlots * 32 * 4;
+    const uint32_t red_bytes = P > 1 ? (uint32_t)nwarps * kSlots * 32 * 4 : 0u;      // no cross-warp sum when a warp owns whole tiles
     L.sbuf_off = (L.red_off + red_bytes + 127u) & ~127u;
     L.ring_off = L.sbuf_off + (uint32_t)nwarps * kScaleBufBytes;
     L.x_off = (L.ring_off + (uint32_t)nwarps * S * chunk + 127u) & ~127u;
@@ -492,35 +492,41 @@ static uint32_t plan_smem(int bits, int K, int P, int G, int S, int cols, LutPla
     return L.x_off + (uint32_t)cols * L.col_stride;
 }
 
-struct Split { int P, G, ctas, S, cols; };
+struct Split { int P, G, slots, ctas, S, cols; };
 
-// Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA, one
-// or two CTAs per SM.  Two smaller CTAs are preferred: with half of an SM's registers and shared memory each, the
-// CTAs of the next launch in the stream (programmatic dependent launch) move in while this launch drains, and their
-// set-up and first copies overlap its tail.  Modelled time of a launch: the larger of what the busiest SM has to issue
-// (tiles x (chunks per tile + a charge per warp for the cross-warp sum, none when a warp owns whole tiles)) and what one
-// warp has to get through on its own; all `want_cols` columns in one pass where shared memory allows.  The constants
-// come from sweeps over (P, G) on 17408x5120, 8192x5120, 5120x17408 and 28672x8192.
+// CTAs of one size class: `slots` of them fit an SM (registers at 80 per thread, shared memory), `ctas` are launched per
+// SM.  (Classes with three or four slots and one of them left free for the first CTAs of the next launch in the stream
+// were measured: the next launch gains nothing from moving in early, and the smaller CTAs lose 15 %.)
+struct SizeClass { int slots, ctas, max_warps; uint32_t smem_cap; };
+static const SizeClass kClasses[] = {
+    {2, 2, 12, kSmemLimitHalf},
+    {1, 1, kMaxWarps, kSmemLimit},
+};
+
+// Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA.
+// Modelled time of a launch, in units of one chunk (8 rows x 1024 weights) of issue work per SM: the larger of what
+// the busiest SM has to issue (tiles x (chunks per tile + a charge per warp for the cross-warp sum, none when a warp
+// owns whole tiles), more when fewer than 16 warps are there to overlap latencies) and what one warp has to get
+// through on its own; all `want_cols` columns in one pass where shared memory allows.  The constants come from sweeps over (P, G) on
+// 17408x5120, 8192x5120, 5120x17408 and 28672x8192.
 static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols)
 {
     const int nslices = (int)lut_slices(K);
     const int64_t ntiles = N / kLutAtomRows;
     double best = 1e300;
-    Split sp = {1, 1, 1, 2, 1};
+    Split sp = {1, 1, 1, 1, 2, 1};
     LutPlan tmp;
-    for (int ctas = 2; ctas >= 1; --ctas) {
-        const int max_warps = ctas == 2 ? 12 : kMaxWarps;
-        const uint32_t smem_cap = ctas == 2 ? kSmemLimitHalf : kSmemLimit;
-        for (int p = 1; p <= nslices && p <= max_warps; ++p) {
+    for (const SizeClass &sc : kClasses) {
+        for (int p = 1; p <= nslices && p <= sc.max_warps; ++p) {
             const int ns_max = (nslices + p - 1) / p;                               // slices of warp 0
-            for (int gg = 1; gg <= kMaxGroups && gg * p <= max_warps; ++gg) {
+            for (int gg = 1; gg <= kMaxGroups && gg * p <= sc.max_warps; ++gg) {
                 int cols = want_cols;
-                while (cols > 1 && plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > smem_cap) --cols;
-                if (plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > smem_cap) continue;
-                const int S = plan_smem(bits, (int)K, p, gg, 3, cols, tmp) <= smem_cap ? 3 : 2;
+                while (cols > 1 && plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) --cols;
+                if (plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) continue;
+                const int S = plan_smem(bits, (int)K, p, gg, 3, cols, tmp) <= sc.smem_cap ? 3 : 2;
                 // CTAs actually launched, CTAs and tiles on the busiest SM, rounds of the busiest group
                 const int64_t need = (ntiles + gg - 1) / gg;
-                const int64_t grid = need < (int64_t)sms * ctas ? need : (int64_t)sms * ctas;
+                const int64_t grid = need < (int64_t)sms * sc.ctas ? need : (int64_t)sms * sc.ctas;
                 const int64_t rounds = (ntiles + grid * gg - 1) / (grid * gg);
                 const double rounds_eff = 0.5 * ((double)rounds + (double)ntiles / (double)(grid * gg));   // SMs finish unevenly, not in lockstep
                 const int64_t ctas_on_sm = (grid + sms - 1) / sms;
@@ -530,8 +536,8 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
                 const double alone = rounds_eff * 8.0 * ns_max;                              // one warp's own chain
                 const int passes = (want_cols + cols - 1) / cols;
                 // ties: two CTAs per SM, then more warps; a second pass over the weights costs a whole launch
-                const double cost = (double)passes * (sm_work > alone ? sm_work : alone) - 1e-3 * ctas * gg * p - (ctas == 2 ? 0.05 : 0.0);
-                if (cost < best) { best = cost; sp = {p, gg, ctas, S, cols}; }
+                const double cost = (double)passes * (sm_work > alone ? sm_work : alone) - 1e-3 * sc.ctas * gg * p - (sc.ctas == 2 ? 0.05 : 0.0);
+                if (cost < best) { best = cost; sp = {p, gg, sc.slots, sc.ctas, S, cols}; }
             }
         }
     }
@@ -539,10 +545,10 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
 }
 
 template <int BITS>
-static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, int threads, int ctas, const LutPlan &L,
+static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, int threads, int slots, const LutPlan &L,
                                uint32_t smem, cudaStream_t stream)
 {
-    if (ctas == 2 && threads <= 384) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    if (slots == 2 && threads <= 384) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
     if (threads <= 768) return launch_one<BITS, 768, 1>(a, b0, cols, grid, threads, L, smem, stream);
     return launch_one<BITS, 1024, 1>(a, b0, cols, grid, threads, L, smem, stream);
 }
@@ -564,12 +570,18 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         sp.P = a.force_P; sp.G = a.force_G;
         sp.S = a.force_S > 0 ? a.force_S : 2;
         sp.cols = want_cols;
-        sp.ctas = (sp.P * sp.G <= 12 && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) <= kSmemLimitHalf) ? 2 : 1;
+        sp.slots = sp.ctas = 1;
+        for (const SizeClass &sc : kClasses)                     // the smallest size class the forced split fits
+            if (sp.P * sp.G <= sc.max_warps && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) <= sc.smem_cap) {
+                sp.slots = sc.slots; sp.ctas = sc.ctas;
+                break;
+            }
         while (sp.cols > 1 && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) > kSmemLimit) --sp.cols;
     } else if (a.force_S > 0) {
         sp.S = a.force_S;
     }
-    const uint32_t smem_cap = sp.ctas == 2 ? kSmemLimitHalf : kSmemLimit;
+    uint32_t smem_cap = kSmemLimit;
+    for (const SizeClass &sc : kClasses) if (sc.slots == sp.slots) smem_cap = sc.smem_cap;
     if (plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) > smem_cap) return cudaErrorInvalidValue;
     const int threads = sp.P * sp.G * 32;
     const int64_t need = ((int64_t)N / kLutAtomRows + sp.G - 1) / sp.G;
@@ -579,8 +591,8 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
     for (int b0 = 0; b0 < B; b0 += sp.cols) {
         const int cols = (B - b0 < sp.cols) ? (B - b0) : sp.cols;
         const uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
-        const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.ctas, L, smem, stream)
-                                            : launch_bits<2>(a, b0, cols, grid, threads, sp.ctas, L, smem, stream);
+        const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.slots, L, smem, stream)
+                                            : launch_bits<2>(a, b0, cols, grid, threads, sp.slots, L, smem, stream);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
