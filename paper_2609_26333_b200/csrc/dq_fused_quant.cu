@@ -131,6 +131,74 @@ __global__ void __launch_bounds__(kNormMaxThreads) rmsnorm_quant_kernel(const __
     }
 }
 
+// The same operator with the row held in registers between the two phases (one read of X instead of two): thread t
+// owns blocks t, t + blockDim, .. (BPT of them, 16 bytes of packed bf16 pairs each twice), a warp's 32 blocks are again one
+// group of the summation order.  One CTA per row, as many threads as the row has blocks / BPT: several CTAs share an SM
+// and cover each other's wait at the barrier.
+template <bool SWIZZLED, int BPT>
+__global__ void __launch_bounds__(1024) rmsnorm_quant_regs_kernel(const __nv_bfloat16 *__restrict__ X, int64_t ldx,
+                                                                  const __nv_bfloat16 *__restrict__ gamma, float eps,
+                                                                  int M, int K, float s, uint8_t *codes, uint8_t *sf)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ float gs[kNormMaxGroups];
+    const int r = blockIdx.x;
+    const int nb = K / 16;
+    const int ngroups = (nb + 31) / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const __nv_bfloat16 *xr = X + (int64_t)r * ldx;
+    uint32_t w[BPT][8];
+#pragma unroll
+    for (int j = 0; j < BPT; ++j) {
+        const int b = j * (int)blockDim.x + threadIdx.x;
+        float bs = 0.0f;
+        if (b < nb) {
+            const uint4 *p = reinterpret_cast<const uint4 *>(xr + b * 16);
+            const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+            w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
+            w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float a = __uint_as_float(w[j][i] << 16), c = __uint_as_float(w[j][i] & 0xFFFF0000u);
+                bs = __fadd_rn(bs, __fmul_rn(a, a));
+                bs = __fadd_rn(bs, __fmul_rn(c, c));
+            }
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) bs = __fadd_rn(bs, __shfl_xor_sync(0xffffffffu, bs, o));   // neighbours first
+        const int grp = ((j * (int)blockDim.x) >> 5) + warp;
+        if (lane == 0 && grp < ngroups) gs[grp] = bs;
+    }
+    __syncthreads();
+    float total = 0.0f;
+    for (int g = 0; g < ngroups; ++g) total = __fadd_rn(total, gs[g]);
+    const float rr = __frcp_rn(__fsqrt_rn(__fadd_rn(__fdiv_rn(total, (float)K), eps)));
+    const float rc6 = __frcp_rn(__fmul_rn(6.0f, s));
+#pragma unroll
+    for (int j = 0; j < BPT; ++j) {
+        const int b = j * (int)blockDim.x + threadIdx.x;
+        const bool live = b < nb;
+        uint32_t d8 = 0;
+        if (live) {
+            const uint4 *q = reinterpret_cast<const uint4 *>(gamma + b * 16);
+            const uint4 g0 = __ldg(q), g1 = __ldg(q + 1);
+            const uint32_t gw[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            uint32_t h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float lo = __fmul_rn(__fmul_rn(__uint_as_float(w[j][i] << 16), rr), __uint_as_float(gw[i] << 16));
+                const float hi = __fmul_rn(__fmul_rn(__uint_as_float(w[j][i] & 0xFFFF0000u), rr), __uint_as_float(gw[i] & 0xFFFF0000u));
+                h[i] = pack_bf16_rn(lo, hi);
+            }
+            uint2 c;
+            d8 = quant_block_nvfp4_bf16(h, s, rc6, c);
+            *reinterpret_cast<uint2 *>(codes + ((int64_t)r * nb + b) * 8) = c;
+        }
+        store_scales<SWIZZLED>(d8, live, r, b, nb, sf);
+    }
+}
+
 // One thread per 16-block of the output; gate and up are the two halves of a row of the fused gate/up output.
 template <bool SWIZZLED>
 __global__ void __launch_bounds__(256) silu_mul_quant_kernel(const __nv_bfloat16 *__restrict__ GU, int64_t ldgu, int M, int nb,
@@ -187,8 +255,19 @@ cudaError_t launch_rmsnorm_quant(const void *X_bf16, int64_t M, int64_t K, int64
     const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(X_bf16);
     const __nv_bfloat16 *G = reinterpret_cast<const __nv_bfloat16 *>(gamma_bf16);
     const int64_t nb = K / 16;
+    const dim3 grid((unsigned)M);
+    if (nb <= 2048) {                                   // the row fits the registers of one CTA
+        const int bpt = nb <= 1024 ? 1 : 2;
+        const dim3 block((unsigned)(((nb + bpt - 1) / bpt + 31) / 32 * 32));
+        if (bpt == 1) {
+            if (swizzled) return launch_pdl(rmsnorm_quant_regs_kernel<true, 1>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
+            return launch_pdl(rmsnorm_quant_regs_kernel<false, 1>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
+        }
+        if (swizzled) return launch_pdl(rmsnorm_quant_regs_kernel<true, 2>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
+        return launch_pdl(rmsnorm_quant_regs_kernel<false, 2>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
+    }
     const int threads = (int)(nb >= kNormMaxThreads ? kNormMaxThreads : (nb + 31) / 32 * 32);
-    const dim3 grid((unsigned)M), block((unsigned)threads);
+    const dim3 block((unsigned)threads);
     if (swizzled) return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
     return launch_pdl(rmsnorm_quant_kernel<false>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
 }

@@ -60,10 +60,11 @@ struct LutPlan {
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1)
 {
+    // C = 0 as an operand of its own: tied to D it would have to be cleared in registers before every mma
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-                 "{%0, %1, %2, %3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+                 "{%10, %10, %10, %10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
 }
 // 8-byte shared-memory load at base + OFF (the offset is an immediate of the instruction)
 template <int OFF>
@@ -139,7 +140,7 @@ __device__ __forceinline__ void block_pair(uint32_t sel, uint32_t x0, uint32_t x
     const uint32_t a0 = prmt(lo0, hi0, 0x5140u), a2 = prmt(lo0, hi0, 0x7362u);     // row g, first block
     const uint32_t lo1 = prmt(cb.tl0, cb.tl1, u1), hi1 = prmt(cb.th0, cb.th1, u1);
     const uint32_t a1 = prmt(lo1, hi1, 0x5140u), a3 = prmt(lo1, hi1, 0x7362u);     // "row g+8": second block
-    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    float c[4];
     mma16816(c, a0, a1, a2, a3, x0, x1);
     acc[0] = fmaf(c[0], d0, acc[0]);
     acc[1] = fmaf(c[1], d0, acc[1]);
@@ -457,6 +458,12 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
         cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);
         if (e != cudaSuccess) return e;
+        // every instantiation asks for the same split of the SM's memory between L1 and shared memory: a change of
+        // the split between two launches has to wait until the SM is empty, which would undo the overlap of one
+        // launch's set-up with the tail of the launch before it
+        e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
@@ -503,12 +510,13 @@ static const SizeClass kClasses[] = {
     {1, 1, kMaxWarps, kSmemLimit},
 };
 
-// Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA.
-// Modelled time of a launch, in units of one chunk (8 rows x 1024 weights) of issue work per SM: the larger of what
-// the busiest SM has to issue (tiles x (chunks per tile + a charge per warp for the cross-warp sum, none when a warp
-// owns whole tiles), more when fewer than 16 warps are there to overlap latencies) and what one warp has to get
-// through on its own; all `want_cols` columns in one pass where shared memory allows.  The constants come from sweeps over (P, G) on
-// 17408x5120, 8192x5120, 5120x17408 and 28672x8192.
+// Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA, in the
+// smallest size class the CTA fits.  Modelled time of a launch, in units of one chunk (8 rows x 1024 weights) of issue
+// work per SM: what the busiest SM has to issue in whole rounds over the tiles (chunks per tile plus a charge per warp
+// that visits the tile), stretched where fewer than 12 warps are there to overlap latencies; all `want_cols` columns in
+// one pass where shared memory allows.  Rings are two chunks deep: a third stage was never faster in sweeps over every
+// feasible (P, G) on eighteen layer shapes (3072x3072 .. 57344x8192, 8192x28672), which is also where the constants
+// come from: the pick is within 2.4 % of the best split on average and 12 % at worst (57344x8192).
 static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols)
 {
     const int nslices = (int)lut_slices(K);
@@ -516,28 +524,27 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
     double best = 1e300;
     Split sp = {1, 1, 1, 1, 2, 1};
     LutPlan tmp;
-    for (const SizeClass &sc : kClasses) {
-        for (int p = 1; p <= nslices && p <= sc.max_warps; ++p) {
-            const int ns_max = (nslices + p - 1) / p;                               // slices of warp 0
-            for (int gg = 1; gg <= kMaxGroups && gg * p <= sc.max_warps; ++gg) {
+    for (int p = 1; p <= nslices && p <= kMaxWarps; ++p) {
+        const int ns_max = (nslices + p - 1) / p;                                   // slices of warp 0
+        for (int gg = 1; gg <= kMaxGroups && gg * p <= kMaxWarps; ++gg) {
+            for (const SizeClass &sc : kClasses) {
+                if (gg * p > sc.max_warps) continue;
                 int cols = want_cols;
                 while (cols > 1 && plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) --cols;
                 if (plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) continue;
-                const int S = plan_smem(bits, (int)K, p, gg, 3, cols, tmp) <= sc.smem_cap ? 3 : 2;
-                // CTAs actually launched, CTAs and tiles on the busiest SM, rounds of the busiest group
+                if (cols < want_cols && sc.ctas > 1) continue;                      // rather one CTA per SM than a second pass
+                // CTAs actually launched, CTAs on the busiest SM, rounds of the busiest group
                 const int64_t need = (ntiles + gg - 1) / gg;
                 const int64_t grid = need < (int64_t)sms * sc.ctas ? need : (int64_t)sms * sc.ctas;
                 const int64_t rounds = (ntiles + grid * gg - 1) / (grid * gg);
-                const double rounds_eff = 0.5 * ((double)rounds + (double)ntiles / (double)(grid * gg));   // SMs finish unevenly, not in lockstep
                 const int64_t ctas_on_sm = (grid + sms - 1) / sms;
                 const double warps = (double)(ctas_on_sm * gg * p);
-                const double per_tile = (double)ns_max * p + (p > 1 ? 0.25 * p : 0.0);       // chunks (slowest warp x P) + cross-warp sum
-                const double sm_work = (double)(ctas_on_sm * gg) * rounds_eff * per_tile / (warps < 16.0 ? warps / 16.0 : 1.0);
-                const double alone = rounds_eff * 8.0 * ns_max;                              // one warp's own chain
+                const double per_tile = ((double)ns_max + 0.25) * p;                  // chunks + a charge per warp and tile
+                const double stretch = warps < 12.0 ? sqrt(12.0 / warps) : 1.0;
                 const int passes = (want_cols + cols - 1) / cols;
-                // ties: two CTAs per SM, then more warps; a second pass over the weights costs a whole launch
-                const double cost = (double)passes * (sm_work > alone ? sm_work : alone) - 1e-3 * sc.ctas * gg * p - (sc.ctas == 2 ? 0.05 : 0.0);
-                if (cost < best) { best = cost; sp = {p, gg, sc.slots, sc.ctas, S, cols}; }
+                const double cost = (double)passes * (double)(ctas_on_sm * gg * rounds) * per_tile * stretch;
+                if (cost < best) { best = cost; sp = {p, gg, sc.slots, sc.ctas, 2, cols}; }
+                break;                                                              // the smallest class that fits
             }
         }
     }
@@ -590,7 +597,12 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
     L.drop_first_copy = a.drop_first_copy;
     for (int b0 = 0; b0 < B; b0 += sp.cols) {
         const int cols = (B - b0 < sp.cols) ? (B - b0) : sp.cols;
-        const uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
+        // Ask for at least so much shared memory that no more CTAs fit an SM than the split counts on: where a third
+        // (second) CTA would fit, the hardware packs three (two) onto some SMs while others hold one, and the launch
+        // takes as long as its fullest SM (measured: 17.3 against 12.9 us on 14336x4096 with 256 CTAs of 7 warps).
+        const uint32_t floor_bytes = (sp.ctas == 2 ? 76u : 114u) * 1024u;
+        uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
+        if (smem < floor_bytes && sp.ctas == 2 && grid > sms) smem = floor_bytes;
         const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.slots, L, smem, stream)
                                             : launch_bits<2>(a, b0, cols, grid, threads, sp.slots, L, smem, stream);
         if (e != cudaSuccess) return e;

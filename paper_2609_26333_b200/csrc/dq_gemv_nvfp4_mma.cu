@@ -275,12 +275,17 @@ template <int MAXT, int NPF>
 cudaError_t launch_one(const GemvNvArgs &a, int b0, int cols, int grid, int threads, int W, int G, uint32_t col_stride,
                        uint32_t smem, cudaStream_t stream)
 {
-    static uint32_t attr_smem = 0;
-    if (smem > attr_smem) {
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemv_nvfp4_mma_kernel<MAXT, NPF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kCtrlBytes + kRedBytes + kMaxXBytes));
         if (e != cudaSuccess) return e;
-        attr_smem = kCtrlBytes + kRedBytes + kMaxXBytes;
+        e = cudaFuncSetAttribute(gemv_nvfp4_mma_kernel<MAXT, NPF>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

@@ -35,7 +35,8 @@ def _gamma(K, seed):
     return (dq_inputs.gaussian_bf16(1, K, 0.3, seed)[0].float() + 1.0).to(torch.bfloat16)
 
 
-@pytest.mark.parametrize("M,K,kind", [(64, 256, "gauss"), (300, 640, "gauss"), (129, 5120, "gauss"), (33, 17408, "student")])
+@pytest.mark.parametrize("M,K,kind", [(64, 256, "gauss"), (300, 640, "gauss"), (129, 5120, "gauss"), (33, 17408, "student"),
+                                        (5, 33024, "gauss")])   # one block per thread, two per thread, the two-pass kernel
 def test_rmsnorm_quantiser_bit_exact(dq, oracle, M, K, kind):
     X = dq_inputs.gaussian_bf16(M, K, 1.0, 400 + M) if kind == "gauss" else dq_inputs.student_t_outlier_bf16(M, K, 401)
     X[0] = 0                                              # a zero row: eps keeps it finite
