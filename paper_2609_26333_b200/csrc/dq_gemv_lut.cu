@@ -513,10 +513,14 @@ static const SizeClass kClasses[] = {
 // Work split: P warps share a tile of 8 rows (each taking 1024-weight slices w, w+P, ..), G such groups per CTA, in the
 // smallest size class the CTA fits.  Modelled time of a launch, in units of one chunk (8 rows x 1024 weights) of issue
 // work per SM: what the busiest SM has to issue in whole rounds over the tiles (chunks per tile plus a charge per warp
-// that visits the tile), stretched where fewer than 12 warps are there to overlap latencies; all `want_cols` columns in
-// one pass where shared memory allows.  Rings are two chunks deep: a third stage was never faster in sweeps over every
-// feasible (P, G) on eighteen layer shapes (3072x3072 .. 57344x8192, 8192x28672), which is also where the constants
-// come from: the pick is within 2.4 % of the best split on average and 12 % at worst (57344x8192).
+// that visits the tile), stretched where fewer than 15 warps share the SM; all `want_cols` columns in one pass where
+// shared memory allows.  Rings are two chunks deep: a third stage was never faster in sweeps over every feasible (P, G)
+// on eighteen layer shapes (3072x3072 .. 57344x8192, 8192x28672), which is also where the constants come from: timed
+// alone, launch after launch of one shape, the pick is within 3 % of the best split on average.  The worst case there
+// (12288x4096, 17 %) is a shape whose best split alone is one CTA of 11 warps per SM; such light launches are avoided
+// on purpose: between a launch of at most 12 warps per SM and one of 15 or more, in either order, about 2 us more pass
+// than between two of a kind (measured on pairs of the 27B-class matrices: 27.8 against 23.3 us for qkv + o), and a
+// token step alternates shapes.
 static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols)
 {
     const int nslices = (int)lut_slices(K);
@@ -540,7 +544,7 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
                 const int64_t ctas_on_sm = (grid + sms - 1) / sms;
                 const double warps = (double)(ctas_on_sm * gg * p);
                 const double per_tile = ((double)ns_max + 0.25) * p;                  // chunks + a charge per warp and tile
-                const double stretch = warps < 12.0 ? sqrt(12.0 / warps) : 1.0;
+                const double stretch = warps < 15.0 ? 15.0 / warps : 1.0;
                 const int passes = (want_cols + cols - 1) / cols;
                 const double cost = (double)passes * (double)(ctas_on_sm * gg * rounds) * per_tile * stretch;
                 if (cost < best) { best = cost; sp = {p, gg, sc.slots, sc.ctas, 2, cols}; }
@@ -555,7 +559,7 @@ template <int BITS>
 static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, int threads, int slots, const LutPlan &L,
                                uint32_t smem, cudaStream_t stream)
 {
-    if (slots == 2 && threads <= 384) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    if (slots == 2 && threads <= 384 && grid > 148) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
     if (threads <= 768) return launch_one<BITS, 768, 1>(a, b0, cols, grid, threads, L, smem, stream);
     return launch_one<BITS, 1024, 1>(a, b0, cols, grid, threads, L, smem, stream);
 }
@@ -600,7 +604,7 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         // Ask for at least so much shared memory that no more CTAs fit an SM than the split counts on: where a third
         // (second) CTA would fit, the hardware packs three (two) onto some SMs while others hold one, and the launch
         // takes as long as its fullest SM (measured: 17.3 against 12.9 us on 14336x4096 with 256 CTAs of 7 warps).
-        const uint32_t floor_bytes = (sp.ctas == 2 ? 76u : 114u) * 1024u;
+        const uint32_t floor_bytes = (grid > sms ? 76u : 114u) * 1024u;      // two CTAs on an SM only where the grid needs them      // two CTAs on an SM only where the grid needs them
         uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
         if (smem < floor_bytes && sp.ctas == 2 && grid > sms) smem = floor_bytes;
         const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.slots, L, smem, stream)
