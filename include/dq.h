@@ -320,7 +320,12 @@ int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsi
  *           a device-side wait budget of `wait_cycles` SM clocks (0 = the default of about two
  *           seconds).  variant 1 additionally leaves out one bulk copy (the first atom of warp 0 of
  *           CTA 0), so that the wait for it runs out after `wait_cycles`: the kernel returns normally,
- *           writes partial output and records DQ_ERR_TIMEOUT for dq_get_status.
+ *           writes partial output and records DQ_ERR_TIMEOUT for dq_get_status.  variant 2 is the
+ *           same kernel as variant 0.  variant 3 (B = 1 only; DQ_ERR_INVALID_ARG where the row is
+ *           too long for its shared-memory layout, about K > 12288) runs the tcgen05 kernel instead:
+ *           levels stored to tensor memory, one tcgen05.mma per 16-weight block, the same exact
+ *           arithmetic; measured slower than the default kernel, it is kept for comparison and is
+ *           not what dq_decode_linear launches.  The three split arguments do not apply to it.
  *   format  DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3: the NVFP4A16 decode; variant 0 = the tensor-core
  *           kernel dq_decode_linear_nvfp4 runs, 1 = the CUDA-core kernel kept for comparison.
  * Other arguments as dq_decode_linear.

@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 OBJ = PKG / "build"
 LIB = PKG / "libdq.so"
-SOURCES = ["dq_api.cu", "dq_pack.cu", "dq_fused_quant.cu", "dq_gemm.cu", "dq_gemm2.cu", "dq_gemv_lut.cu", "dq_gemv_nvfp4.cu", "dq_gemv_nvfp4_mma.cu", "dq_noalloc.cu", "dq_host.cu"]
+SOURCES = ["dq_api.cu", "dq_pack.cu", "dq_fused_quant.cu", "dq_gemm.cu", "dq_gemm2.cu", "dq_gemv_lut.cu", "dq_gemv_lut_tc.cu", "dq_gemv_nvfp4.cu", "dq_gemv_nvfp4_mma.cu", "dq_noalloc.cu", "dq_host.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--ftz=false", "--prec-div=true", "--prec-sqrt=true", "--fmad=true"]
 

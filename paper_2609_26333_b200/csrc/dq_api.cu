@@ -494,7 +494,8 @@ int dq_decode_linear_nvfp4(const dq_weights *w, const void *X_dev, int64_t B, in
 }
 
 static int decode_lut(const dq_weights *w, unsigned format, const void *X_dev, int64_t B, int64_t ldx, void *Y_dev,
-                      int64_t ldy, void *stream, int P, int G, int S, long long wait_cycles, int drop_first_copy = 0)
+                      int64_t ldy, void *stream, int P, int G, int S, long long wait_cycles, int drop_first_copy = 0,
+                      int kernel = 0)
 {
     if (!valid_handle(w) || !X_dev || !Y_dev) return DQ_ERR_INVALID_ARG;
     if (format != DQ_FMT_LUT3 && format != DQ_FMT_LUT2) return DQ_ERR_INVALID_ARG;
@@ -522,6 +523,7 @@ static int decode_lut(const dq_weights *w, unsigned format, const void *X_dev, i
     g.force_S = S;
     g.wait_cycles = wait_cycles;
     g.drop_first_copy = drop_first_copy;
+    g.kernel = kernel;
     const cudaError_t ce = dq::launch_gemv_lut(g, reinterpret_cast<cudaStream_t>(stream));
     if (ce == cudaErrorInvalidValue) return DQ_ERR_INVALID_ARG;
     if (ce != cudaSuccess) return DQ_ERR_CUDA;
@@ -548,8 +550,9 @@ int dq_test_decode_linear(const dq_weights *w, unsigned format, int variant, int
         return decode_nvfp4(w, X_dev, B, ldx, Y_dev, ldy, stream, variant == 0);
     if (warps_per_group < 0 || groups_per_cta < 0 || ring_stages < 0 || ring_stages > 8 || wait_cycles < 0)
         return DQ_ERR_INVALID_ARG;
+    if (variant < 0 || variant > 3) return DQ_ERR_INVALID_ARG;
     return decode_lut(w, format, X_dev, B, ldx, Y_dev, ldy, stream, warps_per_group, groups_per_cta, ring_stages,
-                      wait_cycles, variant == 1 ? 1 : 0);
+                      wait_cycles, variant == 1 ? 1 : 0, variant == 2 ? 1 : variant == 3 ? 2 : 0);
 }
 
 int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, void *scales_dev,

@@ -221,8 +221,12 @@ struct GemvArgs {
     int force_P = 0, force_G = 0, force_S = 0;
     long long wait_cycles = 0;
     int drop_first_copy = 0;                              // one warp's first copy is never requested (its wait must run out)
+    int kernel = 0;                                       // 0 = chosen by the launcher, 1 = mma.sync kernel, 2 = tcgen05 kernel (batch 1)
 };
-cudaError_t launch_gemv_lut(const GemvArgs &args, cudaStream_t stream);     // tensor cores, four batch columns per pass
+cudaError_t launch_gemv_lut(const GemvArgs &args, cudaStream_t stream);     // picks one of the two kernels below
+// tcgen05 kernel (batch 1): number of warpgroups it would run this shape with, 0 where it does not take it
+int gemv_lut_tc_warpgroups(int bits, int64_t N, int64_t K, int64_t B, int sms, bool any_size);
+cudaError_t launch_gemv_lut_tc(const GemvArgs &args, int warpgroups, cudaStream_t stream);
 
 struct GemvNvArgs {
     const uint8_t *codes; const uint8_t *sf;              // NVFP4 view: [N][K/2] codes, MMA-layout scales

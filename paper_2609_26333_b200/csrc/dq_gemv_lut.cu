@@ -573,6 +573,13 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // The tcgen05 kernel runs only where the caller asks for it (test hook): measured, it is the slower of the two
+    // (23.7 against 16.3 us on 17408x5120; its header says why).
+    if (a.kernel == 2) {
+        const int wgs = gemv_lut_tc_warpgroups(a.bits, N, K, B, sms, true);
+        if (wgs == 0) return cudaErrorInvalidValue;
+        return launch_gemv_lut_tc(a, wgs, stream);
+    }
     const int want_cols = B < 4 ? B : 4;
     Split sp = choose_split(a.bits, N, K, sms, want_cols);
     LutPlan L;

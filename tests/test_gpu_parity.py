@@ -601,3 +601,47 @@ def test_host_buffer_entry_points_match_device_calls(dq, oracle):
     with pytest.raises(dq.DQError):
         dq.prefill_linear_host(w, A_host, sa, Y_full[:, :N], staging[:4096])
     _status_ok(dq)
+
+
+# ---- the tcgen05 decode kernel (test-hook variant 3; batch 1): same arithmetic, other machinery ----
+
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(400, 5120, 64), (3072, 12288, 65)])
+def test_decode_tcgen05_kernel_parity(dq, oracle, N, K, seed):
+    """Levels through tensor memory, one tcgen05.mma per 16-weight block: LUT3 and LUT2 against the oracle, on rows
+    that do not fill the last 128-row tile, one to three warpgroups' worth of K, and sparse activations."""
+    W, ref = _layer(oracle, N, K, seed)
+    W2, s2, planes2, scales2 = _lut2_layer(oracle, N, K, seed)
+    assert torch.equal(W, W2)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3 | dq.FMT_LUT2)
+    rows = [dq_inputs.gaussian_bf16(1, K, 1.0, seed + 500)]
+    if K >= 1024:
+        sp = _sparse_patterns(K, seed + 501)
+        rows += [sp[0:1], sp[3:4], sp[10:11], sp[13:14]]
+    for X in rows:
+        Xf = dq_inputs.bf16_to_f32_numpy(X)
+        out = torch.full((1, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+        dq.test_decode_linear(w, dq.FMT_LUT3, X.to(DEV), out=out[:, :N], variant=3)
+        _status_ok(dq)
+        assert torch.all(out[:, N:] == -3.0)
+        Yr, S = oracle.decode_linear(Xf, ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+        check_outputs(_f64(out[:, :N]), Yr, S, f"tcgen05 lut3 decode {N}x{K}")
+        dq.test_decode_linear(w, dq.FMT_LUT2, X.to(DEV), out=out[:, :N], variant=3)
+        _status_ok(dq)
+        Yr, S = oracle.decode_linear_lut2(Xf, planes2, scales2, s2)
+        check_outputs(_f64(out[:, :N]), Yr, S, f"tcgen05 lut2 decode {N}x{K}")
+
+
+def test_decode_tcgen05_kernel_limits(dq):
+    """Batch 1 only, and rows short enough for its shared-memory layout; anything else is refused, not computed."""
+    W = dq_inputs.gaussian_bf16(256, 16384, 0.02, 66)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    X = dq_inputs.gaussian_bf16(2, 16384, 1.0, 67).to(DEV)
+    with pytest.raises(dq.DQError):
+        dq.test_decode_linear(w, dq.FMT_LUT3, X[:1], variant=3)          # K too long
+    W = dq_inputs.gaussian_bf16(256, 1024, 0.02, 68)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3)
+    X = dq_inputs.gaussian_bf16(2, 1024, 1.0, 69).to(DEV)
+    with pytest.raises(dq.DQError):
+        dq.test_decode_linear(w, dq.FMT_LUT3, X, variant=3)              # batch 2
+    dq.test_decode_linear(w, dq.FMT_LUT3, X[:1], variant=3)
+    _status_ok(dq)
