@@ -1,5 +1,5 @@
 // LUT3 / LUT2 weight-only decode (App. C.2 "Kernel specification"; the skinny-batch case the paper leaves open, Sec. 5):
-//   Y[b][n] = bf16( s * sum_blk d_blk(n) * sum_{k in blk} G[idx(n,k)] * X[b][k] ),   up to four batch columns per pass.
+//   Y[b][n] = bf16( s * sum_blk d_blk(n) * sum_{k in blk} G[idx(n,k)] * X[b][k] ),   up to eight batch columns per pass.
 //
 // Arithmetic.  Every product G[idx] * x is exact: the fp16 codebook levels go to the tensor cores unscaled
 // (mma.sync.m16n8k16, fp32 accumulation), the bf16 activations are scaled by one power of two into fp16 (no
@@ -11,8 +11,10 @@
 // Work split.  A row tile is 8 rows.  The 16 rows of the mma's A operand are the 8 rows of the tile against two
 // neighbouring blocks b, b+1; the B operand holds block b of the activations in columns 0-3 (one per batch column)
 // and block b+1 in columns 4-7, so accumulator entries (row g, column c) and (row g+8, column 4+c) are the two
-// halves of one output and the cross terms are dropped.  Lane (g, t) supplies weights 4t .. 4t+3 of both blocks of
-// row g, which is how the device layout stores them (dq_common.cuh).  A group of P warps shares a tile, warp w
+// halves of one output and the cross terms are dropped.  With five to eight batch columns the levels of a lane, once
+// looked up, go through a second mma against the activations of columns 4-7 (template parameter CG, column groups).
+// Lane (g, t) supplies weights 4t .. 4t+3 of both blocks of row g, which is how the device layout stores them
+// (dq_common.cuh).  A group of P warps shares a tile, warp w
 // taking 1024-weight slices w, w+P, .. (P = 1: a warp owns whole tiles and stores its outputs itself; otherwise
 // the last warp of the group to arrive adds the partial tiles in a fixed order); G groups per CTA, one or two
 // CTAs per SM, tiles dealt round robin.
@@ -131,59 +133,82 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 struct Codebook { uint32_t tl0, tl1, th0, th1; };    // low bytes of levels 0-3 / 4-7, high bytes of levels 0-3 / 4-7
 
 // Two neighbouring blocks of the atom (selector word `sel`: low half the first block, high half the second) against
-// their activations xv: one mma, then the two block scales d0, d1 (fp32) on the two block sums.
-__device__ __forceinline__ void block_pair(uint32_t sel, uint32_t x0, uint32_t x1, float d0, float d1, const Codebook &cb,
-                                           float (&acc)[4])
+// their activations: the levels are looked up once, then one mma per group of four batch columns (x0[c], x1[c] its B
+// fragments) and the two block scales d0, d1 (fp32) on the two block sums.
+template <int CG>
+__device__ __forceinline__ void block_pair(uint32_t sel, const uint32_t (&x0)[CG], const uint32_t (&x1)[CG], float d0, float d1,
+                                           const Codebook &cb, float (&acc)[CG][4])
 {
     const uint32_t u1 = sel >> 16;
     const uint32_t lo0 = prmt(cb.tl0, cb.tl1, sel), hi0 = prmt(cb.th0, cb.th1, sel);
     const uint32_t a0 = prmt(lo0, hi0, 0x5140u), a2 = prmt(lo0, hi0, 0x7362u);     // row g, first block
     const uint32_t lo1 = prmt(cb.tl0, cb.tl1, u1), hi1 = prmt(cb.th0, cb.th1, u1);
     const uint32_t a1 = prmt(lo1, hi1, 0x5140u), a3 = prmt(lo1, hi1, 0x7362u);     // "row g+8": second block
-    float c[4];
-    mma16816(c, a0, a1, a2, a3, x0, x1);
-    acc[0] = fmaf(c[0], d0, acc[0]);
-    acc[1] = fmaf(c[1], d0, acc[1]);
-    acc[2] = fmaf(c[2], d1, acc[2]);
-    acc[3] = fmaf(c[3], d1, acc[3]);
+#pragma unroll
+    for (int c = 0; c < CG; ++c) {
+        float d[4];
+        mma16816(d, a0, a1, a2, a3, x0[c], x1[c]);
+        acc[c][0] = fmaf(d[0], d0, acc[c][0]);
+        acc[c][1] = fmaf(d[1], d0, acc[c][1]);
+        acc[c][2] = fmaf(d[2], d1, acc[c][2]);
+        acc[c][3] = fmaf(d[3], d1, acc[c][3]);
+    }
 }
 
 // One word group (32 weights of this lane: four of each of the blocks 8 WI .. 8 WI + 7 of the atom).  The group's
-// activations (this lane's column, block parity and quarter of a block) are 32 contiguous bytes at xa + 256 WI, its eight
-// block scales eight contiguous floats at sa + 32 WI: 16-byte loads serve two mmas each.
-template <int BITS, int WI>
-__device__ __forceinline__ void group_dot(const uint32_t (&w)[BITS], uint32_t xa, uint32_t sa, const Codebook &cb,
-                                          float (&acc)[4])
+// activations (this lane's column of column group c, block parity and quarter of a block) are 32 contiguous bytes at
+// xa[c] + 256 WI, its eight block scales eight contiguous floats at sa + 32 WI: 16-byte loads serve two mmas each.
+template <int BITS, int WI, int CG>
+__device__ __forceinline__ void group_dot(const uint32_t (&w)[BITS], const uint32_t (&xa)[CG], uint32_t sa, const Codebook &cb,
+                                          float (&acc)[CG][4])
 {
     uint32_t sel[4];
     lut_selectors<BITS>(w, sel);
-    const uint4 xA = lds_v4_at<WI * 256>(xa), xB = lds_v4_at<WI * 256 + 16>(xa);
+    uint4 xA[CG], xB[CG];
+#pragma unroll
+    for (int c = 0; c < CG; ++c) {
+        xA[c] = lds_v4_at<WI * 256>(xa[c]);
+        xB[c] = lds_v4_at<WI * 256 + 16>(xa[c]);
+    }
     const float4 dA = lds_v4f_at<WI * 32>(sa), dB = lds_v4f_at<WI * 32 + 16>(sa);
-    block_pair(sel[0], xA.x, xA.y, dA.x, dA.y, cb, acc);
-    block_pair(sel[1], xA.z, xA.w, dA.z, dA.w, cb, acc);
-    block_pair(sel[2], xB.x, xB.y, dB.x, dB.y, cb, acc);
-    block_pair(sel[3], xB.z, xB.w, dB.z, dB.w, cb, acc);
+    uint32_t p0[CG], p1[CG];
+#pragma unroll
+    for (int c = 0; c < CG; ++c) { p0[c] = xA[c].x; p1[c] = xA[c].y; }
+    block_pair<CG>(sel[0], p0, p1, dA.x, dA.y, cb, acc);
+#pragma unroll
+    for (int c = 0; c < CG; ++c) { p0[c] = xA[c].z; p1[c] = xA[c].w; }
+    block_pair<CG>(sel[1], p0, p1, dA.z, dA.w, cb, acc);
+#pragma unroll
+    for (int c = 0; c < CG; ++c) { p0[c] = xB[c].x; p1[c] = xB[c].y; }
+    block_pair<CG>(sel[2], p0, p1, dB.x, dB.y, cb, acc);
+#pragma unroll
+    for (int c = 0; c < CG; ++c) { p0[c] = xB[c].z; p1[c] = xB[c].w; }
+    block_pair<CG>(sel[3], p0, p1, dB.z, dB.w, cb, acc);
 }
 
-// One atom of this lane's row: BITS index words x 4 word groups, against the fp16 activations at shared address xa
-// (this lane's column and block parity; layout in the kernel) and the row's 32 block scales as fp32 at shared address sa.
-template <int BITS>
-__device__ __forceinline__ void atom_dot(const uint4 (&pw)[BITS], uint32_t xa, uint32_t sa, const Codebook &cb,
-                                         float (&acc)[4])
+// One atom of this lane's row: BITS index words x 4 word groups, against the fp16 activations at shared addresses xa[c]
+// + xoff (this lane's column of every column group and block parity; layout in the kernel) and the row's 32 block
+// scales as fp32 at shared address sa.
+template <int BITS, int CG>
+__device__ __forceinline__ void atom_dot(const uint4 (&pw)[BITS], const uint32_t (&xlane)[CG], uint32_t xoff, uint32_t sa,
+                                         const Codebook &cb, float (&acc)[CG][4])
 {
+    uint32_t xa[CG];
+#pragma unroll
+    for (int c = 0; c < CG; ++c) xa[c] = xlane[c] + xoff;      // xoff is 0 or one atom: folded where it is 0
     uint32_t w[BITS];
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].x;
-    group_dot<BITS, 0>(w, xa, sa, cb, acc);
+    group_dot<BITS, 0, CG>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].y;
-    group_dot<BITS, 1>(w, xa, sa, cb, acc);
+    group_dot<BITS, 1, CG>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].z;
-    group_dot<BITS, 2>(w, xa, sa, cb, acc);
+    group_dot<BITS, 2, CG>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].w;
-    group_dot<BITS, 3>(w, xa, sa, cb, acc);
+    group_dot<BITS, 3, CG>(w, xa, sa, cb, acc);
 }
 
 // Activations of one column in shared memory, fp16.  An atom (512 weights, 32 blocks) takes 1024 bytes ordered
@@ -204,7 +229,7 @@ __device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t addr)
 }
 __device__ __forceinline__ void fence_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
 
-template <int BITS, int MAXT, int MINB>
+template <int BITS, int MAXT, int MINB, int CG>
 __global__ void __launch_bounds__(MAXT, MINB)
 gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
                 const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
@@ -327,10 +352,15 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     }
     __syncthreads();
     const float out_scale = s_w * xinv;
-    // B operand of this lane: column g % 4 (column 0 where the pass has fewer), block parity g / 4, weights 4t .. 4t+3
-    const int colsel = ((g & 3) < cols) ? (g & 3) : 0;
-    const uint32_t xlane = win0 + L.x_off + (uint32_t)colsel * L.col_stride + (uint32_t)(g >> 2) * 128u + (uint32_t)t * 32u +
-                           (uint32_t)w * (kLutSlice * 2u);
+    // B operand of this lane in column group c: column 4c + g % 4 (column 0 where the pass has fewer), block parity g / 4,
+    // weights 4t .. 4t+3
+    uint32_t xlane[CG];
+#pragma unroll
+    for (int c = 0; c < CG; ++c) {
+        const int colsel = (4 * c + (g & 3) < cols) ? 4 * c + (g & 3) : 0;
+        xlane[c] = win0 + L.x_off + (uint32_t)colsel * L.col_stride + (uint32_t)(g >> 2) * 128u + (uint32_t)t * 32u +
+                   (uint32_t)w * (kLutSlice * 2u);
+    }
     const uint32_t lane_plane = (uint32_t)lane * 16u;
     // this warp's fp32 scale buffer: 8 rows x 32 blocks; lane l converts bytes 8 l .. 8 l + 7 of the atom's scale bytes
     // (row l / 4, blocks 8 (l % 4) ..), which land at float 8 l of the buffer: row-major like the bytes
@@ -344,9 +374,10 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     uint32_t phase = 0;
     int tile = first;
     for (int it = 0; tile < ntiles; ++it, tile += stride) {
-        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        uint32_t xa = xlane;
-        for (int sl = 0; sl < ns; ++sl, xa += (uint32_t)P * (kLutSlice * 2u)) {
+        float acc[CG][4];
+#pragma unroll
+        for (int c = 0; c < CG; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0f;
+        for (int sl = 0; sl < ns; ++sl) {
             // one lane polls (with back-off) so that waiting warps do not flood the shared-memory pipe; after a wait
             // that ran out every warp keeps walking the same iterations without touching data
             if (ok) {
@@ -368,7 +399,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
-                atom_dot<BITS>(pw, xa, srow, cb, acc);
+                atom_dot<BITS, CG>(pw, xlane, 0u, srow, cb, acc);
                 pw[0] = lds_v4_at<(int)kAtom>(base + lane_plane);
                 pw[1] = lds_v4_at<(int)kAtom + 512>(base + lane_plane);
                 if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(base + lane_plane);
@@ -382,19 +413,31 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
-                atom_dot<BITS>(pw, xa + kLutAtomK * 2u, srow, cb, acc);
+                atom_dot<BITS, CG>(pw, xlane, kLutAtomK * 2u, srow, cb, acc);
             }
             if (++stage == S) { stage = 0; phase ^= 1u; }
+#pragma unroll
+            for (int c = 0; c < CG; ++c) xlane[c] += (uint32_t)P * (kLutSlice * 2u);      // this warp's next slice
         }
+#pragma unroll
+        for (int c = 0; c < CG; ++c) xlane[c] -= (uint32_t)(ns * P) * (kLutSlice * 2u);   // back to its first slice
         // halves of an output: (row g, column c) in lanes t < 2 and (row g + 8, column 4 + c) in lanes t >= 2
-        const float v0 = acc[0] + __shfl_xor_sync(0xffffffffu, acc[2], 2);
-        const float v1 = acc[1] + __shfl_xor_sync(0xffffffffu, acc[3], 2);
+        float v0[CG], v1[CG];
+#pragma unroll
+        for (int c = 0; c < CG; ++c) {
+            v0[c] = acc[c][0] + __shfl_xor_sync(0xffffffffu, acc[c][2], 2);
+            v1[c] = acc[c][1] + __shfl_xor_sync(0xffffffffu, acc[c][3], 2);
+        }
         if (P == 1) {
-            // the warp owns the whole tile: lanes t < 2 hold (row g, columns 2t, 2t+1)
+            // the warp owns the whole tile: lanes t < 2 hold (row g, columns 4c + 2t, 4c + 2t + 1) of column group c
             if (ok && t < 2) {
                 const int row = tile * kLutAtomRows + g;
-                if (2 * t < cols) Y[(int64_t)(b0 + 2 * t) * ldy + row] = __float2bfloat16_rn(v0 * out_scale);
-                if (2 * t + 1 < cols) Y[(int64_t)(b0 + 2 * t + 1) * ldy + row] = __float2bfloat16_rn(v1 * out_scale);
+#pragma unroll
+                for (int c = 0; c < CG; ++c) {
+                    const int col = 4 * c + 2 * t;
+                    if (col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(v0[c] * out_scale);
+                    if (col + 1 < cols) Y[(int64_t)(b0 + col + 1) * ldy + row] = __float2bfloat16_rn(v1[c] * out_scale);
+                }
             }
             continue;
         }
@@ -417,18 +460,25 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
             }
             ok = __shfl_sync(0xffffffffu, good, 0) != 0;
         }
-        float *rbuf = red + (size_t)((grp * kSlots + slot) * P) * 32;
-        if (t < 2) *reinterpret_cast<float2 *>(rbuf + w * 32 + g * 4 + 2 * t) = make_float2(v0, v1);
+        float *rbuf = red + (size_t)((grp * kSlots + slot) * P) * (32 * CG);        // [warp][column group][row 8][column 4]
+        if (t < 2) {
+#pragma unroll
+            for (int c = 0; c < CG; ++c)
+                *reinterpret_cast<float2 *>(rbuf + w * (32 * CG) + c * 32 + g * 4 + 2 * t) = make_float2(v0[c], v1[c]);
+        }
         __syncwarp();
         int prev = 0;
         if (lane == 0) { fence_cta(); prev = atomicAdd(cnt, 1); }
         prev = __shfl_sync(0xffffffffu, prev, 0);
         if (prev == P - 1) {
             fence_cta();
-            float tot = 0.0f;
-            for (int ww = 0; ww < P; ++ww) tot += *reinterpret_cast<const volatile float *>(rbuf + ww * 32 + lane);
-            const int col = lane & 3, row = tile * kLutAtomRows + (lane >> 2);
-            if (ok && col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot * out_scale);
+#pragma unroll
+            for (int c = 0; c < CG; ++c) {
+                float tot = 0.0f;
+                for (int ww = 0; ww < P; ++ww) tot += *reinterpret_cast<const volatile float *>(rbuf + ww * (32 * CG) + c * 32 + lane);
+                const int col = 4 * c + (lane & 3), row = tile * kLutAtomRows + (lane >> 2);
+                if (ok && col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot * out_scale);
+            }
             __syncwarp();
             if (lane == 0) {
                 *cnt = 0;
@@ -447,7 +497,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     }
 }
 
-template <int BITS, int MAXT, int MINB>
+template <int BITS, int MAXT, int MINB, int CG>
 cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int threads, const LutPlan &L, uint32_t smem,
                        cudaStream_t stream)
 {
@@ -455,13 +505,13 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         // every instantiation asks for the same split of the SM's memory between L1 and shared memory: a change of
         // the split between two launches has to wait until the SM is empty, which would undo the overlap of one
         // launch's set-up with the tail of the launch before it
-        e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -476,12 +526,16 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_lut_kernel<BITS, MAXT, MINB>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
+    return cudaLaunchKernelEx(&cfg, gemv_lut_kernel<BITS, MAXT, MINB, CG>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
                               (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
                               (int)a.K, L, a.status);
 }
 
 }  // namespace
+
+// column groups (of four batch columns, one mma each) the kernel is instantiated for
+static int col_groups(int cols) { return cols <= 4 ? 1 : 2; }
+constexpr int kMaxCols = 8;      // 16 columns were measured: their activations leave room for 7 warps, no faster than two passes of 8
 
 // Shared-memory map for P x G warps with S ring stages and `cols` activation columns; returns the bytes needed.
 static uint32_t plan_smem(int bits, int K, int P, int G, int S, int cols, LutPlan &L)
@@ -491,7 +545,8 @@ static uint32_t plan_smem(int bits, int K, int P, int G, int S, int cols, LutPla
     L.P = P; L.G = G; L.S = S;
     L.bar_off = 1024;
     L.red_off = 2048;
-    const uint32_t red_bytes = P > 1 ? (uint32_t)nwarps * kSlots * 32 * 4 : 0u;      // no cross-warp sum when a warp owns whole tiles
+    const uint32_t cg = (uint32_t)col_groups(cols);
+    const uint32_t red_bytes = P > 1 ? (uint32_t)nwarps * kSlots * 32 * 4 * cg : 0u;  // no cross-warp sum when a warp owns whole tiles
     L.sbuf_off = (L.red_off + red_bytes + 127u) & ~127u;
     L.ring_off = L.sbuf_off + (uint32_t)nwarps * kScaleBufBytes;
     L.x_off = (L.ring_off + (uint32_t)nwarps * S * chunk + 127u) & ~127u;
@@ -533,7 +588,7 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
         for (int gg = 1; gg <= kMaxGroups && gg * p <= kMaxWarps; ++gg) {
             for (const SizeClass &sc : kClasses) {
                 if (gg * p > sc.max_warps) continue;
-                int cols = want_cols;
+                int cols = want_cols < kMaxCols ? want_cols : kMaxCols;
                 while (cols > 1 && plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) --cols;
                 if (plan_smem(bits, (int)K, p, gg, 2, cols, tmp) > sc.smem_cap) continue;
                 if (cols < want_cols && sc.ctas > 1) continue;                      // rather one CTA per SM than a second pass
@@ -545,8 +600,9 @@ static Split choose_split(int bits, int64_t N, int64_t K, int sms, int want_cols
                 const double warps = (double)(ctas_on_sm * gg * p);
                 const double per_tile = ((double)ns_max + 0.25) * p;                  // chunks + a charge per warp and tile
                 const double stretch = warps < 15.0 ? 15.0 / warps : 1.0;
+                // every further group of four columns adds an mma, four FFMA and its fragment loads to the eight lookups
                 const int passes = (want_cols + cols - 1) / cols;
-                const double cost = (double)passes * (double)(ctas_on_sm * gg * rounds) * per_tile * stretch;
+                const double cost = (double)passes * (1.0 + 0.2 * (col_groups(cols) - 1)) * (double)(ctas_on_sm * gg * rounds) * per_tile * stretch;
                 if (cost < best) { best = cost; sp = {p, gg, sc.slots, sc.ctas, 2, cols}; }
                 break;                                                              // the smallest class that fits
             }
@@ -559,12 +615,20 @@ template <int BITS>
 static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, int threads, int slots, const LutPlan &L,
                                uint32_t smem, cudaStream_t stream)
 {
-    if (slots == 2 && threads <= 384 && grid > 148) return launch_one<BITS, 384, 2>(a, b0, cols, grid, threads, L, smem, stream);
-    if (threads <= 768) return launch_one<BITS, 768, 1>(a, b0, cols, grid, threads, L, smem, stream);
-    return launch_one<BITS, 1024, 1>(a, b0, cols, grid, threads, L, smem, stream);
+    const int cg = col_groups(cols);
+    if (slots == 2 && threads <= 384 && grid > 148) {
+        if (cg == 1) return launch_one<BITS, 384, 2, 1>(a, b0, cols, grid, threads, L, smem, stream);
+        return launch_one<BITS, 384, 2, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    }
+    if (threads <= 768) {
+        if (cg == 1) return launch_one<BITS, 768, 1, 1>(a, b0, cols, grid, threads, L, smem, stream);
+        return launch_one<BITS, 768, 1, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    }
+    if (cg == 1) return launch_one<BITS, 1024, 1, 1>(a, b0, cols, grid, threads, L, smem, stream);
+    return launch_one<BITS, 1024, 1, 2>(a, b0, cols, grid, threads, L, smem, stream);
 }
 
-// up to four columns per pass
+// up to eight columns per pass
 cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
 {
     const int K = (int)a.K, N = (int)a.N, B = (int)a.B;
@@ -580,14 +644,14 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         if (wgs == 0) return cudaErrorInvalidValue;
         return launch_gemv_lut_tc(a, wgs, stream);
     }
-    const int want_cols = B < 4 ? B : 4;
+    const int want_cols = B;                    // the split decides how many of them one pass takes
     Split sp = choose_split(a.bits, N, K, sms, want_cols);
     LutPlan L;
     if (a.force_P > 0 && a.force_G > 0) {
         if (a.force_P * a.force_G > 32 || a.force_G > kMaxGroups) return cudaErrorInvalidValue;
         sp.P = a.force_P; sp.G = a.force_G;
         sp.S = a.force_S > 0 ? a.force_S : 2;
-        sp.cols = want_cols;
+        sp.cols = want_cols < 8 ? want_cols : 8;                 // every instantiation takes two column groups
         sp.slots = sp.ctas = 1;
         for (const SizeClass &sc : kClasses)                     // the smallest size class the forced split fits
             if (sp.P * sp.G <= sc.max_warps && plan_smem(a.bits, K, sp.P, sp.G, sp.S, sp.cols, L) <= sc.smem_cap) {
@@ -611,9 +675,8 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         // Ask for at least so much shared memory that no more CTAs fit an SM than the split counts on: where a third
         // (second) CTA would fit, the hardware packs three (two) onto some SMs while others hold one, and the launch
         // takes as long as its fullest SM (measured: 17.3 against 12.9 us on 14336x4096 with 256 CTAs of 7 warps).
-        const uint32_t floor_bytes = (grid > sms ? 76u : 114u) * 1024u;      // two CTAs on an SM only where the grid needs them      // two CTAs on an SM only where the grid needs them
         uint32_t smem = L.x_off + (uint32_t)cols * L.col_stride;
-        if (smem < floor_bytes && sp.ctas == 2 && grid > sms) smem = floor_bytes;
+        if (sp.ctas == 2 && grid > sms && smem < 76u * 1024u) smem = 76u * 1024u;
         const cudaError_t e = (a.bits == 3) ? launch_bits<3>(a, b0, cols, grid, threads, sp.slots, L, smem, stream)
                                             : launch_bits<2>(a, b0, cols, grid, threads, sp.slots, L, smem, stream);
         if (e != cudaSuccess) return e;
