@@ -471,6 +471,11 @@ def main():
     d_nv_ms = token_loop_ms(dq.decode_linear_nvfp4)
     # and on the LUT2 weights (2.5 bit per weight)
     d_l2_ms = token_loop_ms(dq.decode_linear_lut2)
+    # the tcgen05 variant of the LUT3 decode (levels through tensor memory; not what dq_decode_linear launches), where its
+    # shared-memory layout takes the row length and the batch is 1
+    d_tc_ms = None
+    if B == 1 and K <= 12288 and not args.no_b2b:
+        d_tc_ms = token_loop_ms(lambda w, X, out: dq.test_decode_linear(w, dq.FMT_LUT3, X, out=out, variant=3))
 
     # ---- measured ceilings (outside the timed region): the GEMM kernel's MMA issue sequence alone, and a
     #      read-only 128-bit streaming pass over the packed copies
@@ -638,6 +643,11 @@ def main():
                                     "frac": l2_bytes / (d_l2_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                                     "ms": d_l2_ms, "timing": "back-to-back launches replayed from one CUDA graph",
                                     "peak_source": f"{peaks['source']} copy bandwidth"}
+    if d_tc_ms:
+        line["roofline_decode"]["tcgen05_variant"] = {"kernel": "gemv_lut_tc_kernel<3>", "ms": d_tc_ms,
+                                                      "achieved": dec_bytes / (d_tc_ms * 1e-3) / 1e9,
+                                                      "frac": dec_bytes / (d_tc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                      "timing": "back-to-back launches replayed from one CUDA graph (test hook)"}
     if fused:
         line["fused_activation_stage"] = fused
     if e2e:
