@@ -282,9 +282,6 @@ cudaError_t launch_one(const GemvNvArgs &a, int b0, int cols, int grid, int thre
         cudaError_t e = cudaFuncSetAttribute(gemv_nvfp4_mma_kernel<MAXT, NPF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kCtrlBytes + kRedBytes + kMaxXBytes));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(gemv_nvfp4_mma_kernel<MAXT, NPF>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 (int)cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
