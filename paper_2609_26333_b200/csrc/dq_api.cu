@@ -66,6 +66,15 @@ bool on_handle_device(const dq_weights *w)
 
 // Prefill workspace: NVFP4 activations (codes, MMA-layout scales); for a handle that stores only
 // LUT3 the NVFP4 view of the weights (codes, MMA-layout scales) follows, rebuilt on every call.
+}  // namespace
+
+namespace dq {
+// for the entry points that live in other files: is this a live handle whose buffers are on the current device?
+bool handle_on_current_device(const dq_weights *w) { return valid_handle(w) && on_handle_device(w); }
+}  // namespace dq
+
+namespace {
+
 struct WsLayout { size_t a_sf = 0, w_codes = 0, w_sf = 0, w_sf_bytes = 0, total = 0; };
 bool has_nvfp4_view(const dq_weights *w) { return (w->formats & (DQ_FMT_NVFP4 | DQ_FMT_NVFP4_FROM_LUT3)) != 0; }
 WsLayout ws_layout(const dq_weights *w, int64_t M)

@@ -161,6 +161,8 @@ __host__ __device__ inline size_t sf_swizzled_offset(int64_t r, int64_t b, int64
 // Device status word: [0] = dq_status, [1] = detail.
 struct StatusWord { int status; int detail; };
 
+bool handle_on_current_device(const dq_weights *w);      // defined beside the handle (dq_api.cu)
+
 // ---- launchers (each enqueues on `stream`, returns a cudaError_t) ----
 cudaError_t launch_pack_header(PackedHeader *hdr, const uint16_t *codebook_f16_host, cudaStream_t stream);
 cudaError_t launch_absmax(const void *W, int w_dtype, int64_t N, int64_t K, int64_t ldw, PackedHeader *hdr,

@@ -54,6 +54,7 @@ extern "C" int dq_prefill_linear_static(const dq_weights *w, const void *A_dev, 
     st = dq_weights_shape(w, &N, &K, nullptr);
     if (st != DQ_OK) return st;
     // Everything dq_prefill_linear would reject is rejected here, before any work is put on the stream.
+    if (!dq::handle_on_current_device(w)) return DQ_ERR_INVALID_ARG;
     if (!A_dev || !Y_dev || !(act_global_scale > 0.0f) || !(act_global_scale <= 3.0e38f)) return DQ_ERR_INVALID_ARG;
     if (lda < K || ldy < N || lda % 8 != 0 || ldy % 8 != 0 || reinterpret_cast<uintptr_t>(A_dev) % 16 != 0 ||
         reinterpret_cast<uintptr_t>(Y_dev) % 16 != 0)
