@@ -135,7 +135,8 @@ struct Codebook { uint32_t tl0, tl1, th0, th1; };    // low bytes of levels 0-3 
 // Two neighbouring blocks of the atom (selector word `sel`: low half the first block, high half the second) against
 // their activations: the levels are looked up once, then one mma per group of four batch columns (x0[c], x1[c] its B
 // fragments) and the two block scales d0, d1 (fp32) on the two block sums.
-template <int CG>
+// (ONE: a single batch column; the odd accumulator columns are never read and are not kept up.)
+template <int CG, bool ONE>
 __device__ __forceinline__ void block_pair(uint32_t sel, const uint32_t (&x0)[CG], const uint32_t (&x1)[CG], float d0, float d1,
                                            const Codebook &cb, float (&acc)[CG][4])
 {
@@ -149,16 +150,16 @@ __device__ __forceinline__ void block_pair(uint32_t sel, const uint32_t (&x0)[CG
         float d[4];
         mma16816(d, a0, a1, a2, a3, x0[c], x1[c]);
         acc[c][0] = fmaf(d[0], d0, acc[c][0]);
-        acc[c][1] = fmaf(d[1], d0, acc[c][1]);
+        if (!ONE) acc[c][1] = fmaf(d[1], d0, acc[c][1]);
         acc[c][2] = fmaf(d[2], d1, acc[c][2]);
-        acc[c][3] = fmaf(d[3], d1, acc[c][3]);
+        if (!ONE) acc[c][3] = fmaf(d[3], d1, acc[c][3]);
     }
 }
 
 // One word group (32 weights of this lane: four of each of the blocks 8 WI .. 8 WI + 7 of the atom).  The group's
 // activations (this lane's column of column group c, block parity and quarter of a block) are 32 contiguous bytes at
 // xa[c] + 256 WI, its eight block scales eight contiguous floats at sa + 32 WI: 16-byte loads serve two mmas each.
-template <int BITS, int WI, int CG>
+template <int BITS, int WI, int CG, bool ONE>
 __device__ __forceinline__ void group_dot(const uint32_t (&w)[BITS], const uint32_t (&xa)[CG], uint32_t sa, const Codebook &cb,
                                           float (&acc)[CG][4])
 {
@@ -174,22 +175,22 @@ __device__ __forceinline__ void group_dot(const uint32_t (&w)[BITS], const uint3
     uint32_t p0[CG], p1[CG];
 #pragma unroll
     for (int c = 0; c < CG; ++c) { p0[c] = xA[c].x; p1[c] = xA[c].y; }
-    block_pair<CG>(sel[0], p0, p1, dA.x, dA.y, cb, acc);
+    block_pair<CG, ONE>(sel[0], p0, p1, dA.x, dA.y, cb, acc);
 #pragma unroll
     for (int c = 0; c < CG; ++c) { p0[c] = xA[c].z; p1[c] = xA[c].w; }
-    block_pair<CG>(sel[1], p0, p1, dA.z, dA.w, cb, acc);
+    block_pair<CG, ONE>(sel[1], p0, p1, dA.z, dA.w, cb, acc);
 #pragma unroll
     for (int c = 0; c < CG; ++c) { p0[c] = xB[c].x; p1[c] = xB[c].y; }
-    block_pair<CG>(sel[2], p0, p1, dB.x, dB.y, cb, acc);
+    block_pair<CG, ONE>(sel[2], p0, p1, dB.x, dB.y, cb, acc);
 #pragma unroll
     for (int c = 0; c < CG; ++c) { p0[c] = xB[c].z; p1[c] = xB[c].w; }
-    block_pair<CG>(sel[3], p0, p1, dB.z, dB.w, cb, acc);
+    block_pair<CG, ONE>(sel[3], p0, p1, dB.z, dB.w, cb, acc);
 }
 
 // One atom of this lane's row: BITS index words x 4 word groups, against the fp16 activations at shared addresses xa[c]
 // + xoff (this lane's column of every column group and block parity; layout in the kernel) and the row's 32 block
 // scales as fp32 at shared address sa.
-template <int BITS, int CG>
+template <int BITS, int CG, bool ONE>
 __device__ __forceinline__ void atom_dot(const uint4 (&pw)[BITS], const uint32_t (&xlane)[CG], uint32_t xoff, uint32_t sa,
                                          const Codebook &cb, float (&acc)[CG][4])
 {
@@ -199,16 +200,16 @@ __device__ __forceinline__ void atom_dot(const uint4 (&pw)[BITS], const uint32_t
     uint32_t w[BITS];
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].x;
-    group_dot<BITS, 0, CG>(w, xa, sa, cb, acc);
+    group_dot<BITS, 0, CG, ONE>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].y;
-    group_dot<BITS, 1, CG>(w, xa, sa, cb, acc);
+    group_dot<BITS, 1, CG, ONE>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].z;
-    group_dot<BITS, 2, CG>(w, xa, sa, cb, acc);
+    group_dot<BITS, 2, CG, ONE>(w, xa, sa, cb, acc);
 #pragma unroll
     for (int p = 0; p < BITS; ++p) w[p] = pw[p].w;
-    group_dot<BITS, 3, CG>(w, xa, sa, cb, acc);
+    group_dot<BITS, 3, CG, ONE>(w, xa, sa, cb, acc);
 }
 
 // Activations of one column in shared memory, fp16.  An atom (512 weights, 32 blocks) takes 1024 bytes ordered
@@ -229,7 +230,7 @@ __device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t addr)
 }
 __device__ __forceinline__ void fence_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
 
-template <int BITS, int MAXT, int MINB, int CG>
+template <int BITS, int MAXT, int MINB, int CG, bool ONE>
 __global__ void __launch_bounds__(MAXT, MINB)
 gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
                 const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
@@ -399,7 +400,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
-                atom_dot<BITS, CG>(pw, xlane, 0u, srow, cb, acc);
+                atom_dot<BITS, CG, ONE>(pw, xlane, 0u, srow, cb, acc);
                 pw[0] = lds_v4_at<(int)kAtom>(base + lane_plane);
                 pw[1] = lds_v4_at<(int)kAtom + 512>(base + lane_plane);
                 if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(base + lane_plane);
@@ -413,7 +414,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
-                atom_dot<BITS, CG>(pw, xlane, kLutAtomK * 2u, srow, cb, acc);
+                atom_dot<BITS, CG, ONE>(pw, xlane, kLutAtomK * 2u, srow, cb, acc);
             }
             if (++stage == S) { stage = 0; phase ^= 1u; }
 #pragma unroll
@@ -497,7 +498,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     }
 }
 
-template <int BITS, int MAXT, int MINB, int CG>
+template <int BITS, int MAXT, int MINB, int CG, bool ONE>
 cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int threads, const LutPlan &L, uint32_t smem,
                        cudaStream_t stream)
 {
@@ -505,13 +506,13 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG, ONE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         // every instantiation asks for the same split of the SM's memory between L1 and shared memory: a change of
         // the split between two launches has to wait until the SM is empty, which would undo the overlap of one
         // launch's set-up with the tail of the launch before it
-        e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        e = cudaFuncSetAttribute(gemv_lut_kernel<BITS, MAXT, MINB, CG, ONE>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -526,7 +527,7 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_lut_kernel<BITS, MAXT, MINB, CG>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
+    return cudaLaunchKernelEx(&cfg, gemv_lut_kernel<BITS, MAXT, MINB, CG, ONE>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
                               (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N,
                               (int)a.K, L, a.status);
 }
@@ -617,15 +618,19 @@ static cudaError_t launch_bits(const GemvArgs &a, int b0, int cols, int grid, in
 {
     const int cg = col_groups(cols);
     if (slots == 2 && threads <= 384 && grid > 148) {
-        if (cg == 1) return launch_one<BITS, 384, 2, 1>(a, b0, cols, grid, threads, L, smem, stream);
-        return launch_one<BITS, 384, 2, 2>(a, b0, cols, grid, threads, L, smem, stream);
+        // a single column with at most 8 warps per CTA: the variant that keeps up two of the four accumulator columns
+        // (it needs more than 80 registers to gain from that)
+        if (cols == 1 && threads <= 256) return launch_one<BITS, 256, 2, 1, true>(a, b0, cols, grid, threads, L, smem, stream);
+        if (cg == 1) return launch_one<BITS, 384, 2, 1, false>(a, b0, cols, grid, threads, L, smem, stream);
+        return launch_one<BITS, 384, 2, 2, false>(a, b0, cols, grid, threads, L, smem, stream);
     }
+    if (cols == 1 && threads <= 640) return launch_one<BITS, 640, 1, 1, true>(a, b0, cols, grid, threads, L, smem, stream);
     if (threads <= 768) {
-        if (cg == 1) return launch_one<BITS, 768, 1, 1>(a, b0, cols, grid, threads, L, smem, stream);
-        return launch_one<BITS, 768, 1, 2>(a, b0, cols, grid, threads, L, smem, stream);
+        if (cg == 1) return launch_one<BITS, 768, 1, 1, false>(a, b0, cols, grid, threads, L, smem, stream);
+        return launch_one<BITS, 768, 1, 2, false>(a, b0, cols, grid, threads, L, smem, stream);
     }
-    if (cg == 1) return launch_one<BITS, 1024, 1, 1>(a, b0, cols, grid, threads, L, smem, stream);
-    return launch_one<BITS, 1024, 1, 2>(a, b0, cols, grid, threads, L, smem, stream);
+    if (cg == 1) return launch_one<BITS, 1024, 1, 1, false>(a, b0, cols, grid, threads, L, smem, stream);
+    return launch_one<BITS, 1024, 1, 2, false>(a, b0, cols, grid, threads, L, smem, stream);
 }
 
 // up to eight columns per pass
