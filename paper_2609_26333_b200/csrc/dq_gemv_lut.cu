@@ -43,7 +43,7 @@ constexpr int kSlots = 4;                         // cross-warp reduction slots 
 constexpr uint32_t kSmemLimit = 227 * 1024;
 constexpr uint32_t kSmemLimitHalf = 113 * 1024;   // two CTAs per SM
 constexpr int kMaxWarps = 24;
-constexpr int kMaxGroups = 12;
+constexpr int kMaxGroups = 16;
 constexpr uint32_t kScaleBufBytes = 1152;         // per warp: 8 rows x 36 floats (32 block scales + 4 of padding)
 
 // shared-memory map (byte offsets from the start of dynamic shared memory) and work split, filled in by the launcher
@@ -243,7 +243,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw);
     int *sync_words = reinterpret_cast<int *>(smem_raw + 64);                           // [G][kSlots] x (generation, count)
-    float *xmax_s = reinterpret_cast<float *>(smem_raw + 512);                          // 32 per-warp maxima
+    float *xmax_s = reinterpret_cast<float *>(smem_raw + 640);                          // 32 per-warp maxima
     float *red = reinterpret_cast<float *>(smem_raw + L.red_off);
 
     const int lane = threadIdx.x & 31;
