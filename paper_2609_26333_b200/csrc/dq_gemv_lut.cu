@@ -106,22 +106,6 @@ __device__ __forceinline__ float4 lds_v4f_at(uint32_t base)
     return v;
 }
 
-// bounded mbarrier wait with back-off between polls
-__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long budget)
-{
-    if (tc::mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t it = 0;
-    while (true) {
-        __nanosleep(20);
-        if (tc::mbar_try(bar, parity)) return true;
-        if ((++it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > budget) { *abort_flag = 1; return false; }
-        }
-    }
-}
-
 // byte permute, selector taken as it is (nibbles with the top bit clear select bytes 0-7 of {a, b})
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
@@ -277,26 +261,34 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     auto tile_base = [&](int tile) {                           // chunk (tile, slice w)
         return lut + (((size_t)(tile >> 1) * nslices + w) * 4u + (size_t)(tile & 1) * 2u) * kAtom;
     };
-    // producer state (lane 0): next chunk to request
+    // Producer state: next chunk to request, its ring stage and barrier.  Every lane keeps it (the arithmetic is uniform),
+    // lane 0 issues: fence, expected bytes and copy are predicated instructions, not a divergent branch.
     const uint8_t *psrc = tile_base(first);
-    int pslice = 0, ptile = (ns > 0) ? first : ntiles, pstage = 0;       // ptile >= ntiles: nothing left to request
+    int pslice = 0, ptile = (ns > 0) ? first : ntiles;                   // ptile >= ntiles: nothing left to request
+    uint32_t pdst = ring0, pbar = bars0;
+    const uint32_t ring_end = ring0 + (uint32_t)S * kChunk;
     auto advance = [&]() {
         if (++pslice == ns) { pslice = 0; ptile += stride; psrc = tile_base(ptile); }
         else psrc += slice_step;
-        if (++pstage == S) pstage = 0;
+        pdst += kChunk;
+        pbar += 8u;
+        if (pdst == ring_end) { pdst = ring0; pbar = bars0; }
     };
-    auto issue_next = [&]() {
-        tc::mbar_expect_tx(bars0 + 8u * pstage, kChunk);
-        tc::bulk_load(ring0 + (uint32_t)pstage * kChunk, psrc, kChunk, bars0 + 8u * pstage);
+    auto issue_next = [&](bool skip_copy) {
+        const uint32_t doit = (lane == 0 && ptile < ntiles && !skip_copy) ? 1u : 0u;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %0, 0;\n\t"
+            "@p fence.proxy.async.shared::cta;\n\t"
+            "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t"
+            "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%3], [%4], %2, [%1];\n\t}"
+            ::"r"(doit), "r"(pbar), "r"(kChunk), "r"(pdst), "l"(psrc) : "memory");
         advance();
     };
     // The weights are constant data: start streaming before waiting for the kernel ahead of this one.
-    if (lane == 0) {
+    {
         const bool drop = L.drop_first_copy && blockIdx.x == 0 && warp == 0;
-        for (int i = 0; i < S && ptile < ntiles; ++i) {
-            if (drop && i == 0) advance();                      // test hook: this chunk is never requested
-            else issue_next();
-        }
+        for (int i = 0; i < S && ptile < ntiles; ++i) issue_next(drop && i == 0);    // test hook: the dropped chunk is never requested
     }
     const uint4 cbv = *reinterpret_cast<const uint4 *>(BITS == 3 ? hdr->lut_prmt : hdr->lut2_prmt);
     const Codebook cb = {cbv.x, cbv.y, cbv.z, cbv.w};
@@ -370,8 +362,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
     const uint32_t swr = sbuf + (uint32_t)(lane >> 2) * 144u + (uint32_t)(lane & 3) * 32u;
     const uint32_t sync0 = win0 + 64u + (uint32_t)grp * kSlots * 8u;
 
-    bool ok = true;
-    int stage = 0;
+    uint32_t cbase = ring0, cbar = bars0;                     // consumer's ring stage and its barrier
     uint32_t phase = 0;
     int tile = first;
     for (int it = 0; tile < ntiles; ++it, tile += stride) {
@@ -379,44 +370,48 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
 #pragma unroll
         for (int c = 0; c < CG; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0f;
         for (int sl = 0; sl < ns; ++sl) {
-            // one lane polls (with back-off) so that waiting warps do not flood the shared-memory pipe; after a wait
-            // that ran out every warp keeps walking the same iterations without touching data
-            if (ok) {
-                uint32_t good = 1;
-                if (lane == 0) good = ring_wait(bars0 + 8u * stage, phase, abort_flag, L.wait_cycles) ? 1u : 0u;
-                ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+            // The chunk is normally there already.  Otherwise poll with back-off; a wait that runs out ends the kernel
+            // for this warp (the others find the flag in their own waits).
+            if (!__any_sync(0xffffffffu, tc::mbar_try(cbar, phase))) {
+                const long long t0 = clock64();
+                bool got = false;
+                while (true) {
+                    __nanosleep(32);
+                    got = __any_sync(0xffffffffu, tc::mbar_try(cbar, phase));
+                    if (got) break;
+                    if (__any_sync(0xffffffffu, *abort_flag != 0 || clock64() - t0 > L.wait_cycles)) break;
+                }
+                if (!got) { *abort_flag = 1; goto give_up; }
             }
-            if (ok) {
-                const uint32_t base = ring0 + (uint32_t)stage * kChunk;
+            {
                 uint4 pw[BITS];
                 uint2 s8;
                 // atom 0: index words to registers; the warp converts the atom's 256 block scales to fp32 once (8 per
                 // lane) and parks them in its scale buffer, from which every lane reads its row's
-                pw[0] = lds_v4_at<0>(base + lane_plane);
-                pw[1] = lds_v4_at<512>(base + lane_plane);
-                if (BITS == 3) pw[BITS - 1] = lds_v4_at<1024>(base + lane_plane);
-                s8 = lds_v2_at<(int)kPlanes>(base + (uint32_t)lane * 8u);
+                pw[0] = lds_v4_at<0>(cbase + lane_plane);
+                pw[1] = lds_v4_at<512>(cbase + lane_plane);
+                if (BITS == 3) pw[BITS - 1] = lds_v4_at<1024>(cbase + lane_plane);
+                s8 = lds_v2_at<(int)kPlanes>(cbase + (uint32_t)lane * 8u);
                 __syncwarp();                                          // everybody is done with the buffer's last contents
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
                 atom_dot<BITS, CG, ONE>(pw, xlane, 0u, srow, cb, acc);
-                pw[0] = lds_v4_at<(int)kAtom>(base + lane_plane);
-                pw[1] = lds_v4_at<(int)kAtom + 512>(base + lane_plane);
-                if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(base + lane_plane);
-                s8 = lds_v2_at<(int)(kAtom + kPlanes)>(base + (uint32_t)lane * 8u);
+                pw[0] = lds_v4_at<(int)kAtom>(cbase + lane_plane);
+                pw[1] = lds_v4_at<(int)kAtom + 512>(cbase + lane_plane);
+                if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(cbase + lane_plane);
+                s8 = lds_v2_at<(int)(kAtom + kPlanes)>(cbase + (uint32_t)lane * 8u);
                 // the stage is in registers: refill it with the chunk S steps ahead
                 __syncwarp();
-                if (lane == 0 && ptile < ntiles) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue_next();
-                }
+                issue_next(false);
                 sts_v4f(swr, e4m3x4_to_f32(s8.x));
                 sts_v4f(swr + 16u, e4m3x4_to_f32(s8.y));
                 __syncwarp();
                 atom_dot<BITS, CG, ONE>(pw, xlane, kLutAtomK * 2u, srow, cb, acc);
             }
-            if (++stage == S) { stage = 0; phase ^= 1u; }
+            cbase += kChunk;
+            cbar += 8u;
+            if (cbase == ring_end) { cbase = ring0; cbar = bars0; phase ^= 1u; }
 #pragma unroll
             for (int c = 0; c < CG; ++c) xlane[c] += (uint32_t)P * (kLutSlice * 2u);      // this warp's next slice
         }
@@ -431,7 +426,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
         }
         if (P == 1) {
             // the warp owns the whole tile: lanes t < 2 hold (row g, columns 4c + 2t, 4c + 2t + 1) of column group c
-            if (ok && t < 2) {
+            if (t < 2) {
                 const int row = tile * kLutAtomRows + g;
 #pragma unroll
                 for (int c = 0; c < CG; ++c) {
@@ -446,7 +441,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
         const int slot = it & (kSlots - 1);
         const uint32_t gen_addr = sync0 + (uint32_t)slot * 8u;
         int *cnt = sync_words + (grp * kSlots + slot) * 2 + 1;
-        if (ok) {
+        {
             uint32_t good = 1;
             if (lane == 0) {
                 const uint32_t want = (uint32_t)(it / kSlots);
@@ -459,7 +454,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                     }
                 }
             }
-            ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+            if (__shfl_sync(0xffffffffu, good, 0) == 0) goto give_up;
         }
         float *rbuf = red + (size_t)((grp * kSlots + slot) * P) * (32 * CG);        // [warp][column group][row 8][column 4]
         if (t < 2) {
@@ -478,7 +473,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
                 float tot = 0.0f;
                 for (int ww = 0; ww < P; ++ww) tot += *reinterpret_cast<const volatile float *>(rbuf + ww * (32 * CG) + c * 32 + lane);
                 const int col = 4 * c + (lane & 3), row = tile * kLutAtomRows + (lane >> 2);
-                if (ok && col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot * out_scale);
+                if (col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(tot * out_scale);
             }
             __syncwarp();
             if (lane == 0) {
@@ -488,6 +483,7 @@ gemv_lut_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict_
             }
         }
     }
+give_up:
     if (*abort_flag) {
         // a wait ran out: let copies in flight land before the CTA's shared memory is handed on, then report
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
