@@ -576,6 +576,33 @@ def test_calls_replay_from_a_cuda_graph(dq, oracle):
     check_outputs(_f64(Y), Yr, S, "graph replay prefill")
 
 
+def test_one_handle_serves_several_streams_at_once(dq, oracle):
+    """A handle is immutable after packing: prefill calls (each with its own workspace) and decode calls issued on
+    three streams at the same time give what the same calls give one after the other, bit for bit."""
+    M, N, K = 640, 2048, 2048
+    W, _ = _layer(oracle, N, K, 75)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4 | dq.FMT_LUT3 | dq.FMT_LUT2)
+    sa = 4.0 / 2688.0
+    streams = [torch.cuda.Stream(device=DEV) for _ in range(3)]
+    A = [dq_inputs.gaussian_bf16(M, K, 1.0, 760 + i).to(DEV) for i in range(3)]
+    X = [dq_inputs.gaussian_bf16(3, K, 1.0, 770 + i).to(DEV) for i in range(3)]
+    wss = [dq.alloc_workspace(dq.prefill_workspace_bytes(w, M), DEV) for _ in range(3)]
+    want = [(dq.prefill_linear(w, A[i], sa, workspace=wss[i]), dq.decode_linear(w, X[i]), dq.decode_linear_lut2(w, X[i]),
+             dq.decode_linear_nvfp4(w, X[i])) for i in range(3)]
+    torch.cuda.synchronize()
+    got = [None] * 3
+    for rep in range(4):                                   # several rounds so that the launches really interleave
+        for i, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                got[i] = (dq.prefill_linear(w, A[i], sa, workspace=wss[i], stream=st), dq.decode_linear(w, X[i], stream=st),
+                          dq.decode_linear_lut2(w, X[i], stream=st), dq.decode_linear_nvfp4(w, X[i], stream=st))
+    torch.cuda.synchronize()
+    _status_ok(dq)
+    for i in range(3):
+        for a, b in zip(got[i], want[i]):
+            assert torch.equal(a, b)
+
+
 def test_host_buffer_entry_points_match_device_calls(dq, oracle):
     """Pinned host activations in, host outputs back, copies inside the call (row chunks pipelined over
     three streams): same bits as the device-pointer calls; strided host rows; M not a multiple of a chunk."""
