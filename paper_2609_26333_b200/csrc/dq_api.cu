@@ -559,9 +559,9 @@ int dq_test_decode_linear(const dq_weights *w, unsigned format, int variant, int
         return decode_nvfp4(w, X_dev, B, ldx, Y_dev, ldy, stream, variant == 0);
     if (warps_per_group < 0 || groups_per_cta < 0 || ring_stages < 0 || ring_stages > 8 || wait_cycles < 0)
         return DQ_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 3) return DQ_ERR_INVALID_ARG;
+    if (variant < 0 || variant > 4) return DQ_ERR_INVALID_ARG;
     return decode_lut(w, format, X_dev, B, ldx, Y_dev, ldy, stream, warps_per_group, groups_per_cta, ring_stages,
-                      wait_cycles, variant == 1 ? 1 : 0, variant == 2 ? 1 : variant == 3 ? 2 : 0);
+                      wait_cycles, variant == 1 ? 1 : 0, variant == 2 ? 1 : variant == 3 ? 2 : variant == 4 ? 3 : 0);
 }
 
 int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, void *scales_dev,

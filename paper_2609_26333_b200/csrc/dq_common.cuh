@@ -223,7 +223,7 @@ struct GemvArgs {
     int force_P = 0, force_G = 0, force_S = 0;
     long long wait_cycles = 0;
     int drop_first_copy = 0;                              // one warp's first copy is never requested (its wait must run out)
-    int kernel = 0;                                       // 0 = chosen by the launcher, 1 = mma.sync kernel, 2 = tcgen05 kernel (batch 1)
+    int kernel = 0;                                       // 0 = chosen by the launcher, 1 = mma.sync kernel, 2 = tcgen05 kernel (batch 1), 3 = slice-by-slice kernel (batches above 8)
 };
 cudaError_t launch_gemv_lut(const GemvArgs &args, cudaStream_t stream);     // picks one of the two kernels below
 // tcgen05 kernel (batch 1): number of warpgroups it would run this shape with, 0 where it does not take it

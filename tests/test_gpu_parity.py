@@ -672,3 +672,31 @@ def test_decode_tcgen05_kernel_limits(dq):
         dq.test_decode_linear(w, dq.FMT_LUT3, X, variant=3)              # batch 2
     dq.test_decode_linear(w, dq.FMT_LUT3, X[:1], variant=3)
     _status_ok(dq)
+
+
+# ---- batches above 8: the kernel that walks K slice by slice with 16 or 32 columns a pass (test-hook variant 4) ----
+
+@pytest.mark.parametrize("N,K,seed", DECODE_SHAPES + [(400, 5120, 64)])
+@pytest.mark.parametrize("B", [9, 16, 17, 33, 64])
+def test_decode_wide_batch_kernel_parity(dq, oracle, N, K, seed, B):
+    """LUT3 and LUT2 against the oracle; activations whose slices differ by many binades (every slice has its own
+    power-of-two scale); strided rows and outputs."""
+    W, ref = _layer(oracle, N, K, seed)
+    W2, s2, planes2, scales2 = _lut2_layer(oracle, N, K, seed)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT3 | dq.FMT_LUT2)
+    X = dq_inputs.gaussian_bf16(B, K, 1.0, seed + 600 + B)
+    X[:, : K // 2] *= 2.0 ** 20
+    X[1] = 0
+    Xd = torch.zeros(B, K + 8, dtype=torch.bfloat16, device=DEV)
+    Xd[:, :K] = X.to(DEV)
+    Xf = dq_inputs.bf16_to_f32_numpy(X)
+    out = torch.full((B, N + 8), -3.0, dtype=torch.bfloat16, device=DEV)
+    dq.test_decode_linear(w, dq.FMT_LUT3, Xd[:, :K], out=out[:, :N], variant=4)
+    _status_ok(dq)
+    assert torch.all(out[:, N:] == -3.0)
+    Yr, S = oracle.decode_linear(Xf, ref["lut3_planes"], ref["lut3_scales"], ref["s"])
+    check_outputs(_f64(out[:, :N]), Yr, S, f"wide lut3 decode {B}x{N}x{K}")
+    dq.test_decode_linear(w, dq.FMT_LUT2, Xd[:, :K], out=out[:, :N], variant=4)
+    _status_ok(dq)
+    Yr, S = oracle.decode_linear_lut2(Xf, planes2, scales2, s2)
+    check_outputs(_f64(out[:, :N]), Yr, S, f"wide lut2 decode {B}x{N}x{K}")
