@@ -530,82 +530,101 @@ cudaError_t launch_one(const GemvArgs &a, int b0, int cols, int grid, int thread
 
 
 // ---------------------------------------------------------------------------------------------------------------
-// Batches above 8: 16 or 32 columns in one pass over the weights.  Their activations do not fit shared memory for a
+// Batches above 8: up to 32 columns in one pass over the weights.  Their activations do not fit shared memory for a
 // whole row, so the CTA walks K slice by slice (1024 weights): all warps stage the slice's activations together
 // (largest magnitude of the slice -> power-of-two scale -> fp16; the scale's inverse goes into the block scales of the
 // slice, which keeps every product exact whatever the other slices hold), then every warp contracts the chunk of its
-// own 8-row tile against them: the levels of a word group are looked up once and go through one mma per group of four
-// columns.  A warp owns whole tiles (one per round over the rows); the rings are those of the kernel above.
+// own tile against them.  Here a tile is 16 rows (the two row halves of the device layout side by side): the 16 rows
+// of the mma's A operand are 16 rows of one block, its 8 columns 8 batch columns, so every accumulator entry is an
+// output and a column costs half the mmas and FFMA of the layout above; the levels of a word group are looked up once
+// and go through one mma per block and group of eight columns.  A warp owns whole tiles (one per round over the rows);
+// a ring stage is the four atoms of a tile and slice, one bulk copy.
 struct WidePlan {
     uint32_t bar_off, sbuf_off, ring_off, x_off, col_stride;
     long long wait_cycles;
 };
 
-template <int BITS, int WI, int CG>
-__device__ __forceinline__ void group_dot_wide(const uint32_t (&w)[BITS], uint32_t xa, uint32_t group_stride, uint32_t sa,
-                                               const Codebook &cb, float (&acc)[CG][4])
+// Activations of one column and slice, fp16: an atom (32 blocks) takes 1024 bytes ordered [word group 4][block pair 4]
+// [quarter t 4][block parity 2][4 weights], so that the B fragments lane (., t) needs for a pair of blocks are 16
+// contiguous bytes.  Byte offset of weights 4t .. 4t+3 of block blk (0..63) of the slice:
+__device__ __forceinline__ uint32_t x16_offset(uint32_t blk, uint32_t t)
 {
-    uint32_t sel[4];
-    lut_selectors<BITS>(w, sel);
-    uint32_t a[4][4];
+    return (blk >> 5) * 1024u + ((blk & 31u) >> 3) * 256u + ((blk & 7u) >> 1) * 64u + t * 16u + (blk & 1u) * 8u;
+}
+
+// One word group of two atoms (rows g and g + 8 of the tile): eight blocks, one mma each per group of eight columns.
+template <int BITS, int WI, int CG8>
+__device__ __forceinline__ void group_dot16(const uint32_t (&w0)[BITS], const uint32_t (&w1)[BITS], uint32_t xa, uint32_t group_stride,
+                                            uint32_t sa0, uint32_t sa1, const Codebook &cb, float (&acc)[CG8][4])
+{
+    uint32_t s0[4], s1[4];
+    lut_selectors<BITS>(w0, s0);
+    lut_selectors<BITS>(w1, s1);
+    uint32_t a[8][4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-        const uint32_t u1 = sel[q] >> 16;
-        const uint32_t lo0 = prmt(cb.tl0, cb.tl1, sel[q]), hi0 = prmt(cb.th0, cb.th1, sel[q]);
-        const uint32_t lo1 = prmt(cb.tl0, cb.tl1, u1), hi1 = prmt(cb.th0, cb.th1, u1);
-        a[q][0] = prmt(lo0, hi0, 0x5140u);
-        a[q][1] = prmt(lo1, hi1, 0x5140u);
-        a[q][2] = prmt(lo0, hi0, 0x7362u);
-        a[q][3] = prmt(lo1, hi1, 0x7362u);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t u0 = h ? (s0[q] >> 16) : s0[q], u1 = h ? (s1[q] >> 16) : s1[q];
+            const uint32_t lo0 = prmt(cb.tl0, cb.tl1, u0), hi0 = prmt(cb.th0, cb.th1, u0);
+            const uint32_t lo1 = prmt(cb.tl0, cb.tl1, u1), hi1 = prmt(cb.th0, cb.th1, u1);
+            a[2 * q + h][0] = prmt(lo0, hi0, 0x5140u);       // row g,     weights 4t, 4t+1
+            a[2 * q + h][1] = prmt(lo1, hi1, 0x5140u);       // row g + 8
+            a[2 * q + h][2] = prmt(lo0, hi0, 0x7362u);       // row g,     weights 4t+2, 4t+3
+            a[2 * q + h][3] = prmt(lo1, hi1, 0x7362u);
+        }
     }
-    const float4 dA = lds_v4f_at<WI * 32>(sa), dB = lds_v4f_at<WI * 32 + 16>(sa);
-    const float d[8] = {dA.x, dA.y, dA.z, dA.w, dB.x, dB.y, dB.z, dB.w};
+    const float4 e0 = lds_v4f_at<WI * 32>(sa0), e1 = lds_v4f_at<WI * 32 + 16>(sa0);
+    const float4 f0 = lds_v4f_at<WI * 32>(sa1), f1 = lds_v4f_at<WI * 32 + 16>(sa1);
+    const float dlo[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};     // row g
+    const float dhi[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};     // row g + 8
 #pragma unroll
-    for (int c = 0; c < CG; ++c) {
-        const uint4 xA = lds_v4_at<WI * 256>(xa), xB = lds_v4_at<WI * 256 + 16>(xa);
+    for (int c = 0; c < CG8; ++c) {
+        const uint4 x0 = lds_v4_at<WI * 256>(xa), x1 = lds_v4_at<WI * 256 + 64>(xa);
+        const uint4 x2 = lds_v4_at<WI * 256 + 128>(xa), x3 = lds_v4_at<WI * 256 + 192>(xa);
         xa += group_stride;
-        const uint32_t xs[8] = {xA.x, xA.y, xA.z, xA.w, xB.x, xB.y, xB.z, xB.w};
+        const uint32_t xs[16] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w, x3.x, x3.y, x3.z, x3.w};
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int i = 0; i < 8; ++i) {
             float r[4];
-            mma16816(r, a[q][0], a[q][1], a[q][2], a[q][3], xs[2 * q], xs[2 * q + 1]);
-            acc[c][0] = fmaf(r[0], d[2 * q], acc[c][0]);
-            acc[c][1] = fmaf(r[1], d[2 * q], acc[c][1]);
-            acc[c][2] = fmaf(r[2], d[2 * q + 1], acc[c][2]);
-            acc[c][3] = fmaf(r[3], d[2 * q + 1], acc[c][3]);
+            mma16816(r, a[i][0], a[i][1], a[i][2], a[i][3], xs[2 * i], xs[2 * i + 1]);
+            acc[c][0] = fmaf(r[0], dlo[i], acc[c][0]);
+            acc[c][1] = fmaf(r[1], dlo[i], acc[c][1]);
+            acc[c][2] = fmaf(r[2], dhi[i], acc[c][2]);
+            acc[c][3] = fmaf(r[3], dhi[i], acc[c][3]);
         }
     }
 }
 
-template <int BITS, int CG>
-__device__ __forceinline__ void atom_dot_wide(const uint4 (&pw)[BITS], uint32_t xa, uint32_t group_stride, uint32_t sa,
-                                              const Codebook &cb, float (&acc)[CG][4])
+template <int BITS, int CG8>
+__device__ __forceinline__ void atom_dot16(const uint4 (&pw0)[BITS], const uint4 (&pw1)[BITS], uint32_t xa, uint32_t group_stride,
+                                           uint32_t sa0, uint32_t sa1, const Codebook &cb, float (&acc)[CG8][4])
 {
-    uint32_t w[BITS];
+    uint32_t w0[BITS], w1[BITS];
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) w[p] = pw[p].x;
-    group_dot_wide<BITS, 0, CG>(w, xa, group_stride, sa, cb, acc);
+    for (int p = 0; p < BITS; ++p) { w0[p] = pw0[p].x; w1[p] = pw1[p].x; }
+    group_dot16<BITS, 0, CG8>(w0, w1, xa, group_stride, sa0, sa1, cb, acc);
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) w[p] = pw[p].y;
-    group_dot_wide<BITS, 1, CG>(w, xa, group_stride, sa, cb, acc);
+    for (int p = 0; p < BITS; ++p) { w0[p] = pw0[p].y; w1[p] = pw1[p].y; }
+    group_dot16<BITS, 1, CG8>(w0, w1, xa, group_stride, sa0, sa1, cb, acc);
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) w[p] = pw[p].z;
-    group_dot_wide<BITS, 2, CG>(w, xa, group_stride, sa, cb, acc);
+    for (int p = 0; p < BITS; ++p) { w0[p] = pw0[p].z; w1[p] = pw1[p].z; }
+    group_dot16<BITS, 2, CG8>(w0, w1, xa, group_stride, sa0, sa1, cb, acc);
 #pragma unroll
-    for (int p = 0; p < BITS; ++p) w[p] = pw[p].w;
-    group_dot_wide<BITS, 3, CG>(w, xa, group_stride, sa, cb, acc);
+    for (int p = 0; p < BITS; ++p) { w0[p] = pw0[p].w; w1[p] = pw1[p].w; }
+    group_dot16<BITS, 3, CG8>(w0, w1, xa, group_stride, sa0, sa1, cb, acc);
 }
 
-template <int BITS, int CG>
-__global__ void __launch_bounds__(512, 1)
+template <int BITS, int CG8>
+__global__ void __launch_bounds__(384, 1)
 gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__restrict__ hdr,
                      const __nv_bfloat16 *__restrict__ X, int64_t ldx, int b0, int cols,
                      __nv_bfloat16 *__restrict__ Y, int64_t ldy, int N, int K, WidePlan L, StatusWord *status)
 {
     constexpr uint32_t kAtom = (uint32_t)lut_atom_bytes(BITS);
-    constexpr uint32_t kChunk = 2u * kAtom;
+    constexpr uint32_t kStage = 4u * kAtom;                  // the four atoms of one 16-row tile and slice
     constexpr uint32_t kPlanes = (uint32_t)lut_plane_bytes(BITS);
-    constexpr int kCols = 4 * CG;
+    constexpr int kCols = 8 * CG8;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t win0 = (uint32_t)__cvta_generic_to_shared(smem_raw);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw);
@@ -615,14 +634,14 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     const int G = blockDim.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int nslices = (int)lut_slices(K);
-    const int ntiles = N / kLutAtomRows;
+    const int ntiles = N / 16;
     const int per_round = gridDim.x * G;
     const int rounds = (ntiles + per_round - 1) / per_round;
     const int first = blockIdx.x * G + warp;
 
-    const uint32_t ring0 = win0 + L.ring_off + (uint32_t)warp * 2u * kChunk;
+    const uint32_t ring0 = win0 + L.ring_off + (uint32_t)warp * 2u * kStage;
     const uint32_t bars0 = win0 + L.bar_off + (uint32_t)warp * 16u;
-    const uint32_t ring_end = ring0 + 2u * kChunk;
+    const uint32_t ring_end = ring0 + 2u * kStage;
     if (lane == 0) {
         tc::mbar_init(bars0, 1);
         tc::mbar_init(bars0 + 8u, 1);
@@ -632,11 +651,8 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     if (threadIdx.x == 0) *abort_flag = 0;
     __syncwarp();
 
-    auto tile_base = [&](int tile) {
-        return lut + ((size_t)(tile >> 1) * nslices * 4u + (size_t)(tile & 1) * 2u) * kAtom;
-    };
-    // producer: the chunks of this warp's tiles, slice after slice, round after round
-    const uint8_t *psrc = tile_base(first);
+    // producer: the stages of this warp's tiles, slice after slice, round after round
+    const uint8_t *psrc = lut + (size_t)first * nslices * kStage;
     int pslice = 0, ptile = first;
     uint32_t pdst = ring0, pbar = bars0;
     auto issue_next = [&]() {
@@ -647,10 +663,10 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
             "@p fence.proxy.async.shared::cta;\n\t"
             "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t"
             "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%3], [%4], %2, [%1];\n\t}"
-            ::"r"(doit), "r"(pbar), "r"(kChunk), "r"(pdst), "l"(psrc) : "memory");
-        if (++pslice == nslices) { pslice = 0; ptile += per_round; psrc = tile_base(ptile); }
-        else psrc += 4u * kAtom;
-        pdst += kChunk;
+            ::"r"(doit), "r"(pbar), "r"(kStage), "r"(pdst), "l"(psrc) : "memory");
+        if (++pslice == nslices) { pslice = 0; ptile += per_round; psrc = lut + (size_t)ptile * nslices * kStage; }
+        else psrc += kStage;
+        pdst += kStage;
         pbar += 8u;
         if (pdst == ring_end) { pdst = ring0; pbar = bars0; }
     };
@@ -667,10 +683,12 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     // columns the pass does not have read as zero
     for (int i = threadIdx.x; i < (kCols - cols) * (int)(L.col_stride / 16); i += blockDim.x)
         *reinterpret_cast<uint4 *>(xh + (size_t)cols * L.col_stride + (size_t)i * 16) = make_uint4(0u, 0u, 0u, 0u);
-    const uint32_t xlane = win0 + L.x_off + (uint32_t)(g & 3) * L.col_stride + (uint32_t)(g >> 2) * 128u + (uint32_t)t * 32u;
-    const uint32_t group_stride = 4u * L.col_stride;
+    // B operand of this lane: column g of every group of eight, weights 4t .. 4t+3 of a pair of blocks per 16-byte load
+    const uint32_t xlane = win0 + L.x_off + (uint32_t)g * L.col_stride + (uint32_t)t * 16u;
+    const uint32_t group_stride = 8u * L.col_stride;
     const uint32_t lane_plane = (uint32_t)lane * 16u;
-    const uint32_t sbuf = win0 + L.sbuf_off + (uint32_t)warp * kScaleBufBytes;
+    // fp32 scale buffers of the two atoms (row halves) being worked on
+    const uint32_t sbuf = win0 + L.sbuf_off + (uint32_t)warp * (2u * kScaleBufBytes);
     const uint32_t srow = sbuf + (uint32_t)g * 144u;
     const uint32_t swr = sbuf + (uint32_t)(lane >> 2) * 144u + (uint32_t)(lane & 3) * 32u;
 
@@ -679,15 +697,15 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     const int items = cols * 128;                        // 16-byte pieces of a slice's activations
     for (int r = 0, tile = first; r < rounds; ++r, tile += per_round) {
         const bool active = tile < ntiles;
-        float acc[CG][4];
+        float acc[CG8][4];
 #pragma unroll
-        for (int c = 0; c < CG; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0f;
+        for (int c = 0; c < CG8; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0f;
         for (int sl = 0; sl < nslices; ++sl) {
             // ---- the slice's activations: largest magnitude, power-of-two scale, fp16.  A thread's pieces are loaded in
-            //      one batch (one trip to L2, not one per piece) and stay in registers across the reduction; CTAs too
-            //      small for that read them a second time.
-            constexpr int kBatch = 9;
-            const bool one_batch = items <= (int)blockDim.x * kBatch;
+            //      batches of eight (one trip to L2 per batch, not per piece); what does not fit one batch is read a
+            //      second time after the reduction.
+            constexpr int kBatch = 8;
+            const int nbatch = (items + (int)blockDim.x * kBatch - 1) / ((int)blockDim.x * kBatch);
             uint4 v[kBatch];
             float m = 0.0f;
             auto piece_max = [&](const uint4 &q) {
@@ -696,23 +714,22 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
                 const uint32_t lo = max(max(a0 & 0xFFFFu, a1 & 0xFFFFu), max(a2 & 0xFFFFu, a3 & 0xFFFFu));
                 return __uint_as_float(max(hi, lo) << 16);
             };
-            auto load_piece = [&](int i) {
-                const int c = i >> 7, k8 = sl * 128 + (i & 127);
-                uint4 q = make_uint4(0u, 0u, 0u, 0u);                     // beyond K (a short last slice): zero
-                if (i < items && k8 < K / 8) q = __ldg(reinterpret_cast<const uint4 *>(X + (int64_t)(b0 + c) * ldx) + k8);
-                return q;
-            };
-            if (one_batch) {
+            auto load_batch = [&](int bi) {                                   // eight loads in flight per thread
 #pragma unroll
-                for (int u = 0; u < kBatch; ++u) v[u] = load_piece((int)threadIdx.x + u * (int)blockDim.x);
+                for (int u = 0; u < kBatch; ++u) {
+                    const int i = (bi * kBatch + u) * (int)blockDim.x + (int)threadIdx.x;
+                    const int c = i >> 7, k8 = sl * 128 + (i & 127);
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);                       // beyond K (a short last slice): zero
+                    if (i < items && k8 < K / 8) v[u] = __ldg(reinterpret_cast<const uint4 *>(X + (int64_t)(b0 + c) * ldx) + k8);
+                }
+            };
+            for (int bi = 0; bi < nbatch; ++bi) {
+                load_batch(bi);
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) m = fmaxf(m, piece_max(v[u]));
-            } else {
-                for (int i = threadIdx.x; i < items; i += blockDim.x) m = fmaxf(m, piece_max(load_piece(i)));
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            // (the maxima of the slice before were read before its chunks were worked on: the buffer is free)
             if (lane == 0) xmax_s[(sl & 1) * 16 + warp] = m;
             __syncthreads();                             // maxima there; nobody reads the slice before this one any more
             m = (lane < G) ? xmax_s[(sl & 1) * 16 + lane] : 0.0f;
@@ -722,29 +739,28 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
             ex = max(-100, min(100, ex));
             const float xscale = __uint_as_float((uint32_t)(127 + 14 - ex) << 23);      // 2^(14 - ex)
             const float sscale = __uint_as_float((uint32_t)(127 - 14 + ex) << 23);      // its inverse, into the block scales
-            auto store_piece = [&](int i, const uint4 &q) {
-                if (i >= items) return;
-                const int c = i >> 7, j = i & 127;
-                const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
-                uint32_t h4[4];
+            for (int bi = nbatch - 1; bi >= 0; --bi) {               // the last batch is still in registers
+                if (bi != nbatch - 1) load_batch(bi);
 #pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                    const __half2 h = __floats2half2_rn(__uint_as_float(ww[z] << 16) * xscale, __uint_as_float(ww[z] & 0xFFFF0000u) * xscale);
-                    h4[z] = *reinterpret_cast<const uint32_t *>(&h);
+                for (int u = 0; u < kBatch; ++u) {
+                    const int i = (bi * kBatch + u) * (int)blockDim.x + (int)threadIdx.x;
+                    if (i >= items) continue;
+                    const uint32_t c = (uint32_t)i >> 7, j = (uint32_t)i & 127u;          // piece j: half h of block j / 2
+                    const uint32_t ww[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    uint32_t h4[4];
+#pragma unroll
+                    for (int z = 0; z < 4; ++z) {
+                        const __half2 h = __floats2half2_rn(__uint_as_float(ww[z] << 16) * xscale, __uint_as_float(ww[z] & 0xFFFF0000u) * xscale);
+                        h4[z] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    uint8_t *px = xh + (size_t)c * L.col_stride + x16_offset(j >> 1, (j & 1u) * 2u);
+                    *reinterpret_cast<uint2 *>(px) = make_uint2(h4[0], h4[1]);           // weights 4t .. 4t+3, t = 2h
+                    *reinterpret_cast<uint2 *>(px + 16) = make_uint2(h4[2], h4[3]);      // t = 2h + 1
                 }
-                uint8_t *px = xh + (size_t)c * L.col_stride + x_offset(j);
-                *reinterpret_cast<uint2 *>(px) = make_uint2(h4[0], h4[1]);
-                *reinterpret_cast<uint2 *>(px + 32) = make_uint2(h4[2], h4[3]);
-            };
-            if (one_batch) {
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) store_piece((int)threadIdx.x + u * (int)blockDim.x, v[u]);
-            } else {
-                for (int i = threadIdx.x; i < items; i += blockDim.x) store_piece(i, load_piece(i));
             }
             __syncthreads();
             if (!active) continue;
-            // ---- this warp's chunk of the slice
+            // ---- this warp's stage of the slice
             if (!dead && !__any_sync(0xffffffffu, tc::mbar_try(cbar, phase))) {
                 const long long t0 = clock64();
                 bool got = false;
@@ -757,46 +773,49 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
                 if (!got) { *abort_flag = 1; dead = true; }
             }
             if (!dead) {
-                uint4 pw[BITS];
-                uint2 s8;
-                pw[0] = lds_v4_at<0>(cbase + lane_plane);
-                pw[1] = lds_v4_at<512>(cbase + lane_plane);
-                if (BITS == 3) pw[BITS - 1] = lds_v4_at<1024>(cbase + lane_plane);
-                s8 = lds_v2_at<(int)kPlanes>(cbase + (uint32_t)lane * 8u);
-                __syncwarp();
-                float4 f = e4m3x4_to_f32(s8.x);
-                sts_v4f(swr, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
-                f = e4m3x4_to_f32(s8.y);
-                sts_v4f(swr + 16u, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
-                __syncwarp();
-                atom_dot_wide<BITS, CG>(pw, xlane, group_stride, srow, cb, acc);
-                pw[0] = lds_v4_at<(int)kAtom>(cbase + lane_plane);
-                pw[1] = lds_v4_at<(int)kAtom + 512>(cbase + lane_plane);
-                if (BITS == 3) pw[BITS - 1] = lds_v4_at<(int)kAtom + 1024>(cbase + lane_plane);
-                s8 = lds_v2_at<(int)(kAtom + kPlanes)>(cbase + (uint32_t)lane * 8u);
-                __syncwarp();
-                issue_next();
-                f = e4m3x4_to_f32(s8.x);
-                sts_v4f(swr, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
-                f = e4m3x4_to_f32(s8.y);
-                sts_v4f(swr + 16u, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
-                __syncwarp();
-                atom_dot_wide<BITS, CG>(pw, xlane + kLutAtomK * 2u, group_stride, srow, cb, acc);
-                cbase += kChunk;
+                // atoms of the stage: (row half 0, k half 0), (0, 1), (1, 0), (1, 1)
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {
+                    uint4 pw0[BITS], pw1[BITS];
+                    const uint32_t at0 = cbase + (uint32_t)kh * kAtom, at1 = cbase + (uint32_t)(2 + kh) * kAtom;
+                    pw0[0] = lds_v4_at<0>(at0 + lane_plane);
+                    pw0[1] = lds_v4_at<512>(at0 + lane_plane);
+                    if (BITS == 3) pw0[BITS - 1] = lds_v4_at<1024>(at0 + lane_plane);
+                    pw1[0] = lds_v4_at<0>(at1 + lane_plane);
+                    pw1[1] = lds_v4_at<512>(at1 + lane_plane);
+                    if (BITS == 3) pw1[BITS - 1] = lds_v4_at<1024>(at1 + lane_plane);
+                    const uint2 sa = lds_v2_at<(int)kPlanes>(at0 + (uint32_t)lane * 8u);
+                    const uint2 sb = lds_v2_at<(int)kPlanes>(at1 + (uint32_t)lane * 8u);
+                    __syncwarp();                                  // everybody is done with the buffers' last contents
+                    if (kh == 1) issue_next();                     // the stage is in registers: refill it
+                    float4 f = e4m3x4_to_f32(sa.x);
+                    sts_v4f(swr, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
+                    f = e4m3x4_to_f32(sa.y);
+                    sts_v4f(swr + 16u, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
+                    f = e4m3x4_to_f32(sb.x);
+                    sts_v4f(swr + kScaleBufBytes, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
+                    f = e4m3x4_to_f32(sb.y);
+                    sts_v4f(swr + kScaleBufBytes + 16u, make_float4(f.x * sscale, f.y * sscale, f.z * sscale, f.w * sscale));
+                    __syncwarp();
+                    atom_dot16<BITS, CG8>(pw0, pw1, xlane + (uint32_t)kh * 1024u, group_stride, srow, srow + kScaleBufBytes, cb, acc);
+                }
+                cbase += kStage;
                 cbar += 8u;
                 if (cbase == ring_end) { cbase = ring0; cbar = bars0; phase ^= 1u; }
             }
         }
         if (active && !dead) {
-            // halves of an output: (row g, column c) in lanes t < 2 and (row g + 8, column 4 + c) in lanes t >= 2
+            // lane (g, t) holds rows g and g + 8 of the tile in columns 2t, 2t + 1 of every group of eight
 #pragma unroll
-            for (int c = 0; c < CG; ++c) {
-                const float v0 = acc[c][0] + __shfl_xor_sync(0xffffffffu, acc[c][2], 2);
-                const float v1 = acc[c][1] + __shfl_xor_sync(0xffffffffu, acc[c][3], 2);
-                if (t < 2) {
-                    const int row = tile * kLutAtomRows + g, col = 4 * c + 2 * t;
-                    if (col < cols) Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(v0 * s_w);
-                    if (col + 1 < cols) Y[(int64_t)(b0 + col + 1) * ldy + row] = __float2bfloat16_rn(v1 * s_w);
+            for (int c = 0; c < CG8; ++c) {
+                const int row = tile * 16 + g, col = 8 * c + 2 * t;
+                if (col < cols) {
+                    Y[(int64_t)(b0 + col) * ldy + row] = __float2bfloat16_rn(acc[c][0] * s_w);
+                    Y[(int64_t)(b0 + col) * ldy + row + 8] = __float2bfloat16_rn(acc[c][2] * s_w);
+                }
+                if (col + 1 < cols) {
+                    Y[(int64_t)(b0 + col + 1) * ldy + row] = __float2bfloat16_rn(acc[c][1] * s_w);
+                    Y[(int64_t)(b0 + col + 1) * ldy + row + 8] = __float2bfloat16_rn(acc[c][3] * s_w);
                 }
             }
         }
@@ -810,7 +829,7 @@ gemv_lut_wide_kernel(const uint8_t *__restrict__ lut, const PackedHeader *__rest
     }
 }
 
-template <int BITS, int CG>
+template <int BITS, int CG8>
 cudaError_t launch_wide_one(const GemvArgs &a, int b0, int cols, int grid, int threads, const WidePlan &L, uint32_t smem,
                             cudaStream_t stream)
 {
@@ -818,9 +837,9 @@ cudaError_t launch_wide_one(const GemvArgs &a, int b0, int cols, int grid, int t
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_wide_kernel<BITS, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_wide_kernel<BITS, CG8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(gemv_lut_wide_kernel<BITS, CG>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(gemv_lut_wide_kernel<BITS, CG8>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -834,7 +853,7 @@ cudaError_t launch_wide_one(const GemvArgs &a, int b0, int cols, int grid, int t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_lut_wide_kernel<BITS, CG>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
+    return cudaLaunchKernelEx(&cfg, gemv_lut_wide_kernel<BITS, CG8>, a.lut, a.hdr, reinterpret_cast<const __nv_bfloat16 *>(a.X),
                               (int64_t)a.ldx, b0, cols, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.N, (int)a.K, L,
                               a.status);
 }
@@ -842,28 +861,43 @@ cudaError_t launch_wide_one(const GemvArgs &a, int b0, int cols, int grid, int t
 // all of B in passes of up to 32 columns
 cudaError_t launch_wide(const GemvArgs &a, int sms, cudaStream_t stream)
 {
-    const int64_t ntiles = a.N / kLutAtomRows;
-    int G = (int)((ntiles + sms - 1) / sms);
-    G = G < 4 ? 4 : (G > 15 ? 15 : G);
-    const uint32_t chunk = 2u * (uint32_t)lut_atom_bytes(a.bits);
+    const int64_t ntiles = a.N / 16;
+    const uint32_t stage = 4u * (uint32_t)lut_atom_bytes(a.bits);
+    // Warps per CTA (each owns one 16-row tile per round): as few tiles on the busiest SM as the rounds allow, among
+    // the counts whose rings fit beside 32 columns of a slice; of equals the larger.
+    int G = 4;
+    int64_t best = -1;
+    for (int cand = 4; cand <= 9; ++cand) {
+        const int64_t busiest = ((ntiles + (int64_t)sms * cand - 1) / ((int64_t)sms * cand)) * cand;
+        if (best < 0 || busiest <= best) { best = busiest; G = cand; }
+    }
     WidePlan L;
     L.bar_off = 1024;
     L.sbuf_off = 2048;
-    L.ring_off = L.sbuf_off + (uint32_t)G * kScaleBufBytes;
-    L.x_off = (L.ring_off + (uint32_t)G * 2u * chunk + 127u) & ~127u;
-    L.col_stride = kLutSlice * 2u + 16u;
+    L.ring_off = L.sbuf_off + (uint32_t)G * 2u * kScaleBufBytes;
+    L.x_off = (L.ring_off + (uint32_t)G * 2u * stage + 127u) & ~127u;
+    L.col_stride = kLutSlice * 2u + 64u;                 // 64 mod 128: the 16-byte loads of two columns hit different banks
     L.wait_cycles = a.wait_cycles > 0 ? a.wait_cycles : tc::kWaitBudgetCycles;
     const int64_t need = (ntiles + G - 1) / G;
     const int grid = (int)(need < sms ? need : sms);
     for (int b0 = 0; b0 < (int)a.B;) {
         const int left = (int)a.B - b0;
-        const int cg = left > 16 ? 8 : 4;
-        const int cols = left < 4 * cg ? left : 4 * cg;
-        const uint32_t smem = L.x_off + (uint32_t)(4 * cg) * L.col_stride;
+        const int cg = left > 24 ? 4 : left > 16 ? 3 : left > 8 ? 2 : 1;
+        const int cols = left < 8 * cg ? left : 8 * cg;
+        const uint32_t smem = L.x_off + (uint32_t)(8 * cg) * L.col_stride;
         if (smem > kSmemLimit) return cudaErrorInvalidValue;
-        cudaError_t e;
-        if (a.bits == 3) e = cg == 8 ? launch_wide_one<3, 8>(a, b0, cols, grid, G * 32, L, smem, stream) : launch_wide_one<3, 4>(a, b0, cols, grid, G * 32, L, smem, stream);
-        else e = cg == 8 ? launch_wide_one<2, 8>(a, b0, cols, grid, G * 32, L, smem, stream) : launch_wide_one<2, 4>(a, b0, cols, grid, G * 32, L, smem, stream);
+        cudaError_t e = cudaErrorInvalidValue;
+        if (a.bits == 3) {
+            if (cg == 4) e = launch_wide_one<3, 4>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else if (cg == 3) e = launch_wide_one<3, 3>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else if (cg == 2) e = launch_wide_one<3, 2>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else e = launch_wide_one<3, 1>(a, b0, cols, grid, G * 32, L, smem, stream);
+        } else {
+            if (cg == 4) e = launch_wide_one<2, 4>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else if (cg == 3) e = launch_wide_one<2, 3>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else if (cg == 2) e = launch_wide_one<2, 2>(a, b0, cols, grid, G * 32, L, smem, stream);
+            else e = launch_wide_one<2, 1>(a, b0, cols, grid, G * 32, L, smem, stream);
+        }
         if (e != cudaSuccess) return e;
         b0 += cols;
     }
@@ -987,9 +1021,8 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         if (wgs == 0) return cudaErrorInvalidValue;
         return launch_gemv_lut_tc(a, wgs, stream);
     }
-    // batches above 12 (below, two passes of the kernel above are as fast) on enough rows to give every SM several tiles:
-    // the kernel that walks K slice by slice
-    if ((a.kernel == 3 || (a.kernel == 0 && a.force_P == 0 && B > 12 && (int64_t)N / kLutAtomRows >= (int64_t)sms * 8)))
+    // batches above 8 on enough rows to give every SM several 16-row tiles: the kernel that walks K slice by slice
+    if ((a.kernel == 3 || (a.kernel == 0 && a.force_P == 0 && B > 8 && (int64_t)N / 16 > (int64_t)sms * 6)))
         return launch_wide(a, sms, stream);
     const int want_cols = B;                    // the split decides how many of them one pass takes
     Split sp = choose_split(a.bits, N, K, sms, want_cols);
