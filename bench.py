@@ -448,7 +448,7 @@ def main():
     nb2b = 2 if args.no_b2b else max(50, 3 * copies)
     b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def token_loop_ms(fn):
+    def token_loop_ms(fn, X=X, Yd=Yd):
         for i in range(copies):
             fn(ws[i], X, out=Yd)
         torch.cuda.synchronize()
@@ -471,6 +471,13 @@ def main():
     d_nv_ms = token_loop_ms(dq.decode_linear_nvfp4)
     # and on the LUT2 weights (2.5 bit per weight)
     d_l2_ms = token_loop_ms(dq.decode_linear_lut2)
+    # LUT3 decode at larger batches (skinny GEMM on the same weights): back-to-back launches, ms per launch
+    d_batches = {}
+    if not args.no_b2b:
+        for bb in (2, 4, 8, 16, 32, 64):
+            Xb = torch.randn(bb, K, dtype=torch.float32, device=dev).to(torch.bfloat16)
+            Yb = torch.empty(bb, N, dtype=torch.bfloat16, device=dev)
+            d_batches[str(bb)] = token_loop_ms(dq.decode_linear, Xb, Yb)
     # the tcgen05 variant of the LUT3 decode (levels through tensor memory; not what dq_decode_linear launches), where its
     # shared-memory layout takes the row length and the batch is 1
     d_tc_ms = None
@@ -643,6 +650,8 @@ def main():
                                     "frac": l2_bytes / (d_l2_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                                     "ms": d_l2_ms, "timing": "back-to-back launches replayed from one CUDA graph",
                                     "peak_source": f"{peaks['source']} copy bandwidth"}
+    if d_batches:
+        line["decode"]["back_to_back_ms_by_batch"] = d_batches
     if d_tc_ms:
         line["roofline_decode"]["tcgen05_variant"] = {"kernel": "gemv_lut_tc_kernel<3>", "ms": d_tc_ms,
                                                       "achieved": dec_bytes / (d_tc_ms * 1e-3) / 1e9,
