@@ -34,7 +34,7 @@ CONFIGS = {
     # 8B-class fused QKV
     "c2_qkv8b": LayerConfig("c2_qkv8b", N=6144, K=4096, M=2048, decode_batches=(1, 8), cfg_id=2),
     # 27B-class FFN
-    "c3_gate_up27b": LayerConfig("c3_gate_up27b", N=17408, K=5120, M=8192, decode_batches=(1, 4, 16), cfg_id=3,
+    "c3_gate_up27b": LayerConfig("c3_gate_up27b", N=17408, K=5120, M=8192, decode_batches=(1, 4, 16, 40), cfg_id=3,
                                  matrix_id=0),
     "c3_down27b": LayerConfig("c3_down27b", N=5120, K=17408, M=8192, decode_batches=(1, 4, 16), cfg_id=3,
                               matrix_id=1),
