@@ -163,6 +163,31 @@ int dq_prefill_silu_mul_quantize(const dq_weights *w, const void *GU_dev, int64_
                                  void *stream);
 
 /*
+ * The gate/up projection of a gated FFN with the gating and the next layer's activation quantiser in the GEMM's
+ * epilogue (App. C.1: activation processing fused with the quantiser; Sec. 2.3 prefill path):
+ *   H = bf16( SiLU(G) * U ),  [G | U] = bf16( A^ W_gate_up^T ),   out_workspace <- NVFP4(H) with out_global_scale,
+ * i.e. what dq_prefill_gemm on w_gate_up followed by dq_prefill_silu_mul_quantize for w_down produces, without the
+ * M x 2F bf16 matrix ever going to memory.  Call order for the whole FFN:
+ *   dq_prefill_quantize (or dq_prefill_rmsnorm_quantize) for w_gate_up into `workspace`, this call,
+ *   dq_prefill_gemm(w_down, M, out_global_scale, Y, ldy, out_workspace, ...).
+ * w_gate_up: 2F x K, one tensor (one global scale), with its rows INTERLEAVED so that a 256-row tile holds gate and
+ *   up of the same 128 features: row 256 t + 128 h + 64 p + j (h, p in {0, 1}, j < 64) is the gate (p = 0) or up
+ *   (p = 1) row of feature 128 t + 64 h + j.  The caller permutes the rows before dq_pack_weights; the handle does
+ *   not record the order, and the same handle passed to dq_prefill_gemm gives the columns in this order.
+ * w_down: N_out x F (F a multiple of 128, as every packed K); only its shape, and for a DQ_FMT_LUT3-only handle its
+ *   call-time NVFP4 cast, are used here.  w_gate_up's N must equal 2 * w_down's K, else DQ_ERR_SHAPE.
+ * workspace: the quantised input, as for dq_prefill_gemm(w_gate_up, M, act_global_scale, ...).
+ * out_workspace: at least dq_prefill_workspace_bytes(w_down, M) bytes, 1024-byte aligned, not overlapping
+ *   `workspace` (DQ_ERR_INVALID_ARG); written by this call, then read by dq_prefill_gemm(w_down, ...).
+ * Arithmetic: G and U are rounded to bf16 exactly as dq_prefill_gemm would store them, SiLU and the quantiser are those
+ * of dq_prefill_silu_mul_quantize; for M > 128 codes and scales equal the two-call path bit for bit.
+ */
+int dq_prefill_gemm_silu_mul_quantize(const dq_weights *w_gate_up, int64_t M, float act_global_scale,
+                                      const void *workspace_dev, size_t workspace_bytes,
+                                      const dq_weights *w_down, float out_global_scale,
+                                      void *out_workspace_dev, size_t out_workspace_bytes, void *stream);
+
+/*
  * dq_prefill_linear without a caller-provided workspace.  (The paper has no counterpart: this
  * entry point exists for integration, not for the method.)
  * It is meant for callers that cannot allocate device memory where they call from -- an engine
@@ -299,6 +324,13 @@ int dq_rmsnorm_quantize_activations(const void *X_dev, int64_t M, int64_t K, int
 int dq_silu_mul_quantize_activations(const void *GU_dev, int64_t M, int64_t F, int64_t ldgu,
                                      float act_global_scale, void *codes_dev, void *scales_dev,
                                      void *stream);
+
+/*
+ * Test hook: out[i] = SiLU(g[i]) in fp32 exactly as the gated quantisers evaluate it (dq_prefill_silu_mul_quantize,
+ * dq_prefill_gemm_silu_mul_quantize; App. C.1 fused activation processing), for n bf16 values on the device.  There
+ * are only 65536 inputs, so a test can compare the fixed fp32 sequence with a CPU evaluation for every one of them.
+ */
+int dq_test_silu(const void *g_dev, int64_t n, float *out_dev, void *stream);
 
 /*
  * Reads the library's device status word for the current device (synchronises

@@ -23,8 +23,9 @@ SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights
            "dq_prefill_linear_static",
            "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear",
            "dq_bench_gemm_mma_only", "dq_bench_stream_read",
-           "dq_prefill_rmsnorm_quantize", "dq_prefill_silu_mul_quantize", "dq_rmsnorm_quantize_activations",
-           "dq_silu_mul_quantize_activations", "dq_export_canonical", "dq_import_canonical",
+           "dq_prefill_rmsnorm_quantize", "dq_prefill_silu_mul_quantize", "dq_prefill_gemm_silu_mul_quantize",
+           "dq_rmsnorm_quantize_activations",
+           "dq_silu_mul_quantize_activations", "dq_test_silu", "dq_export_canonical", "dq_import_canonical",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
            "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
@@ -87,6 +88,10 @@ def lib() -> C.CDLL:
         L.dq_prefill_rmsnorm_quantize.argtypes = [vp, vp, i64, i64, vp, C.c_float, C.c_float, vp, sz, vp]
         L.dq_prefill_silu_mul_quantize.restype = C.c_int
         L.dq_prefill_silu_mul_quantize.argtypes = [vp, vp, i64, i64, C.c_float, vp, sz, vp]
+        L.dq_test_silu.restype = C.c_int
+        L.dq_test_silu.argtypes = [vp, i64, vp, vp]
+        L.dq_prefill_gemm_silu_mul_quantize.restype = C.c_int
+        L.dq_prefill_gemm_silu_mul_quantize.argtypes = [vp, i64, C.c_float, vp, sz, vp, C.c_float, vp, sz, vp]
         L.dq_rmsnorm_quantize_activations.restype = C.c_int
         L.dq_rmsnorm_quantize_activations.argtypes = [vp, i64, i64, i64, vp, C.c_float, C.c_float, vp, vp, vp]
         L.dq_silu_mul_quantize_activations.restype = C.c_int
@@ -273,6 +278,34 @@ def prefill_silu_mul_quantize(w: DQWeights, GU: torch.Tensor, act_global_scale: 
            "dq_prefill_silu_mul_quantize")
 
 
+def gate_up_row_order(F: int) -> torch.Tensor:
+    """Row order dq_prefill_gemm_silu_mul_quantize expects of a fused gate/up matrix: entry r of the result is the row
+    of [gate; up] (gate rows 0..F-1, up rows F..2F-1) that goes to row r, i.e. row 256 t + 128 h + 64 p + j holds
+    gate (p = 0) or up (p = 1) of feature 128 t + 64 h + j.  Index arithmetic only."""
+    assert F % 128 == 0
+    r = torch.arange(2 * F)
+    t, h, p, j = r // 256, (r // 128) % 2, (r // 64) % 2, r % 64
+    return p * F + 128 * t + 64 * h + j
+
+
+def prefill_gemm_silu_mul_quantize(w_gate_up: DQWeights, M: int, act_global_scale: float, workspace: torch.Tensor,
+                                   w_down: DQWeights, out_global_scale: float, out_workspace: torch.Tensor, stream=None):
+    """dq_prefill_gemm_silu_mul_quantize: the gate/up GEMM with SiLU(gate) * up and the down projection's activation
+    quantiser in its epilogue; follow with prefill_gemm(w_down, M, out_global_scale, Y, out_workspace)."""
+    _check(lib().dq_prefill_gemm_silu_mul_quantize(w_gate_up.handle, M, float(act_global_scale), workspace.data_ptr(),
+                                                   workspace.numel(), w_down.handle, float(out_global_scale),
+                                                   out_workspace.data_ptr(), out_workspace.numel(), _stream_ptr(stream)),
+           "dq_prefill_gemm_silu_mul_quantize")
+
+
+def test_silu(g: torch.Tensor, stream=None) -> torch.Tensor:
+    """dq_test_silu: the device SiLU of the gated quantisers, value by value (fp32)."""
+    assert g.is_cuda and g.dtype == torch.bfloat16 and g.is_contiguous()
+    out = torch.empty(g.numel(), dtype=torch.float32, device=g.device)
+    _check(lib().dq_test_silu(g.data_ptr(), g.numel(), out.data_ptr(), _stream_ptr(stream)), "dq_test_silu")
+    return out
+
+
 def rmsnorm_quantize_activations(X: torch.Tensor, gamma: torch.Tensor, eps: float, act_global_scale: float, stream=None):
     assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
     M, K = X.shape
@@ -350,6 +383,7 @@ def test_decode_linear(w: DQWeights, fmt: int, X: torch.Tensor, out: torch.Tenso
 
 
 test_decode_linear.__test__ = False      # not a pytest test
+test_silu.__test__ = False
 
 
 def bench_gemm_mma_only(w: DQWeights, M: int, out: torch.Tensor, workspace: torch.Tensor, stream=None):

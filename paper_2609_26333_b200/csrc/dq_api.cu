@@ -437,6 +437,49 @@ int dq_prefill_gemm(const dq_weights *w, int64_t M, float act_global_scale, void
     return prefill_gemm(w, M, act_global_scale, Y_dev, ldy, workspace_dev, workspace_bytes, stream, false);
 }
 
+int dq_prefill_gemm_silu_mul_quantize(const dq_weights *w_gate_up, int64_t M, float act_global_scale,
+                                      const void *workspace_dev, size_t workspace_bytes, const dq_weights *w_down,
+                                      float out_global_scale, void *out_workspace_dev, size_t out_workspace_bytes,
+                                      void *stream)
+{
+    int st = prefill_checks(w_gate_up, M, act_global_scale, workspace_dev, workspace_bytes);
+    if (st != DQ_OK) return st;
+    st = prefill_checks(w_down, M, out_global_scale, out_workspace_dev, out_workspace_bytes);
+    if (st != DQ_OK) return st;
+    if (w_gate_up->N != 2 * w_down->K) return DQ_ERR_SHAPE;
+    {   // the GEMM reads one workspace while its epilogue writes the other
+        const uintptr_t a0 = reinterpret_cast<uintptr_t>(workspace_dev), a1 = a0 + workspace_bytes;
+        const uintptr_t b0 = reinterpret_cast<uintptr_t>(out_workspace_dev), b1 = b0 + out_workspace_bytes;
+        if (a0 < b1 && b0 < a1) return DQ_ERR_INVALID_ARG;
+    }
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    dq::StatusWord *sw = status_word_ptr();
+    if (!sw) return DQ_ERR_CUDA;
+    const uint8_t *ws = reinterpret_cast<const uint8_t *>(workspace_dev);
+    uint8_t *ows = reinterpret_cast<uint8_t *>(out_workspace_dev);
+    const WsLayout L = ws_layout(w_gate_up, M), LO = ws_layout(w_down, M);
+    dq::GemmArgs g;
+    g.a_codes = ws;
+    g.a_sf = ws + L.a_sf;
+    g.w_codes = has_nvfp4_view(w_gate_up) ? w_gate_up->base + w_gate_up->layout.nv_codes_off : ws + L.w_codes;
+    g.w_sf = has_nvfp4_view(w_gate_up) ? w_gate_up->base + w_gate_up->layout.nv_sf_off : ws + L.w_sf;
+    g.hdr = reinterpret_cast<const dq::PackedHeader *>(w_gate_up->base);
+    g.act_scale = act_global_scale;
+    g.Y = nullptr;
+    g.ldy = w_gate_up->N;
+    g.M = M;
+    g.N = w_gate_up->N;
+    g.K = w_gate_up->K;
+    g.status = sw;
+    g.gated_codes = ows;
+    g.gated_sf = ows + LO.a_sf;
+    g.gated_scale = out_global_scale;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (dq::launch_gemm_nvfp4(g, s) != cudaSuccess) return DQ_ERR_CUDA;
+    return prefill_weight_view(w_down, ows, LO, s);
+}
+
 int dq_bench_gemm_mma_only(const dq_weights *w, int64_t M, void *Y_dev, int64_t ldy, const void *workspace_dev,
                            size_t workspace_bytes, void *stream)
 {
@@ -640,6 +683,15 @@ int dq_silu_mul_quantize_activations(const void *GU_dev, int64_t M, int64_t F, i
                                   reinterpret_cast<uint8_t *>(scales_dev), 0, reinterpret_cast<cudaStream_t>(stream)) !=
         cudaSuccess)
         return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_test_silu(const void *g_dev, int64_t n, float *out_dev, void *stream)
+{
+    if (!g_dev || !out_dev || n < 1) return DQ_ERR_INVALID_ARG;
+    int st = check_arch();
+    if (st != DQ_OK) return st;
+    if (dq::launch_silu_probe(g_dev, n, out_dev, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
 

@@ -196,6 +196,7 @@ cudaError_t launch_rmsnorm_quant(const void *X_bf16, int64_t M, int64_t K, int64
                                  float act_scale, uint8_t *codes, uint8_t *sf, int swizzled, cudaStream_t stream);
 cudaError_t launch_silu_mul_quant(const void *GU_bf16, int64_t M, int64_t F, int64_t ldgu, float act_scale, uint8_t *codes,
                                   uint8_t *sf, int swizzled, cudaStream_t stream);
+cudaError_t launch_silu_probe(const void *g_bf16, int64_t n, float *out, cudaStream_t stream);
 
 struct GemmArgs {
     const uint8_t *a_codes;  const uint8_t *a_sf;      // activations: [M][K/2], MMA scale layout
@@ -206,6 +207,9 @@ struct GemmArgs {
     int64_t M, N, K;
     StatusWord *status;
     bool mma_only = false;   // measurement: MMA issue sequence only (pair kernel; no loads, scale copies or stores)
+    // gated epilogue (pair kernel only): W is a fused gate/up matrix with interleaved rows, and instead of Y the kernel
+    // writes NVFP4(bf16(SiLU(gate) * up)) with input scale gated_scale: codes [M][N/4], block scales in the MMA's layout
+    uint8_t *gated_codes = nullptr; uint8_t *gated_sf = nullptr; float gated_scale = 0.0f;
 };
 cudaError_t launch_gemm_nvfp4(const GemmArgs &args, cudaStream_t stream);
 cudaError_t launch_gemm_nvfp4_pair(const GemmArgs &args, void *encode_fn, cudaStream_t stream);

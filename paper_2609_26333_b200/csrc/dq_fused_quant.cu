@@ -22,33 +22,6 @@ namespace {
 constexpr int kNormMaxThreads = 256;        // one thread per 16-block where the row has that few
 constexpr int kNormMaxGroups = 256;          // groups of 32 blocks per row: K <= 131072
 
-__device__ __forceinline__ float silu_f32(float g)
-{
-    const float L_HI = 1.4426950216293335f, L_LO = 1.925963033500256e-08f;      // log2(e) = L_HI + L_LO
-    const float t = __fmul_rn(g, -L_HI);
-    const float n = rintf(fminf(fmaxf(t, -126.0f), 126.0f));
-    float f = __fmaf_rn(g, -L_HI, -n);
-    f = __fmaf_rn(g, -L_LO, f);
-    f = fminf(fmaxf(f, -1.0f), 1.0f);
-    float p = 1.5252733804059841e-05f;
-    p = __fmaf_rn(p, f, 0.00015403530393381608f);
-    p = __fmaf_rn(p, f, 0.0013333558146428443f);
-    p = __fmaf_rn(p, f, 0.009618129107628477f);
-    p = __fmaf_rn(p, f, 0.05550410866482158f);
-    p = __fmaf_rn(p, f, 0.2402265069591007f);
-    p = __fmaf_rn(p, f, 0.6931471805599453f);
-    p = __fmaf_rn(p, f, 1.0f);
-    const float e = __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
-    return __fdiv_rn(g, __fadd_rn(1.0f, e));
-}
-
-__device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
 // scale bytes of the four blocks of one 64-wide k atom (lanes 4q .. 4q+3) -> one 32-bit store
 template <bool SWIZZLED>
 __device__ __forceinline__ void store_scales(uint32_t d8, bool live, int r, int b, int nb, uint8_t *sf)
@@ -219,16 +192,21 @@ __global__ void __launch_bounds__(256) silu_mul_quant_kernel(const __nv_bfloat16
         const uint32_t uw[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
         uint32_t h[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float lo = __fmul_rn(silu_f32(__uint_as_float(gw[i] << 16)), __uint_as_float(uw[i] << 16));
-            const float hi = __fmul_rn(silu_f32(__uint_as_float(gw[i] & 0xFFFF0000u)), __uint_as_float(uw[i] & 0xFFFF0000u));
-            h[i] = pack_bf16_rn(lo, hi);
-        }
+        for (int i = 0; i < 8; ++i) h[i] = silu_mul_bf16x2(gw[i], uw[i]);
         uint2 c;
         d8 = quant_block_nvfp4_bf16(h, s, rc6, c);
         *reinterpret_cast<uint2 *>(codes + ((int64_t)r * nb + b) * 8) = c;
     }
     store_scales<SWIZZLED>(d8, live, r, b, nb, sf);
+}
+
+// test hook: the SiLU the kernels above and the gated GEMM epilogue evaluate, value by value
+__global__ void silu_probe_kernel(const __nv_bfloat16 *__restrict__ g, int64_t n, float *__restrict__ out)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float x = __bfloat162float(g[i]);
+    out[i] = silu_f32(x);
 }
 
 template <typename Kern, typename... Args>
@@ -270,6 +248,12 @@ cudaError_t launch_rmsnorm_quant(const void *X_bf16, int64_t M, int64_t K, int64
     const dim3 block((unsigned)threads);
     if (swizzled) return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
     return launch_pdl(rmsnorm_quant_kernel<false>, grid, block, stream, X, ldx, G, eps, (int)M, (int)K, act_scale, codes, sf);
+}
+
+cudaError_t launch_silu_probe(const void *g_bf16, int64_t n, float *out, cudaStream_t stream)
+{
+    silu_probe_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16 *>(g_bf16), n, out);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_silu_mul_quant(const void *GU_bf16, int64_t M, int64_t F, int64_t ldgu, float act_scale, uint8_t *codes,

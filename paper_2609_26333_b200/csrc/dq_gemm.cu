@@ -265,7 +265,8 @@ cudaError_t launch_gemm_nvfp4(const GemmArgs &a, cudaStream_t stream)
 {
     if (gemm_init_driver_api() != 0) return cudaErrorNotSupported;
     // more than one 128-row block: CTA pairs share the W tile; otherwise a lone CTA per tile
-    if (a.M > BM) return launch_gemm_nvfp4_pair(a, reinterpret_cast<void *>(g_encode), stream);
+    // (the gated epilogue exists in the pair kernel only)
+    if (a.M > BM || a.gated_codes) return launch_gemm_nvfp4_pair(a, reinterpret_cast<void *>(g_encode), stream);
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;

@@ -19,9 +19,18 @@
 //                 convert, swizzled smem staging and TMA stores overlap the next tile's MMAs
 // Every wait is bounded; a wait that runs out sets DQ_ERR_TIMEOUT and all roles
 // of both CTAs leave through the common exit.
+//
+// Gated epilogue (EPI = 1; App. C.1: activation processing fused with the activation quantiser).  For the fused
+// gate/up projection of a gated FFN whose weight rows are stored interleaved -- row 256 t + 128 h + 64 p + j holds
+// gate (p = 0) or up (p = 1) of feature 128 t + 64 h + j -- every epilogue thread finds gate and up of 64 features
+// of its row in its own registers.  It rounds both to bf16 (what the plain epilogue would have stored), forms
+// bf16(SiLU(gate) * up), quantises the four 16-blocks to NVFP4 with the next layer's static input scale and writes
+// 32 bytes of codes and one 32-bit word of block scales straight into the workspace of the down projection: the
+// M x 2F bf16 matrix is neither written nor read back.
 #include <cuda.h>
 
 #include "dq_common.cuh"
+#include "dq_quant.cuh"
 #include "dq_tcgen05.cuh"
 
 namespace dq {
@@ -53,7 +62,9 @@ struct Cfg {
     static constexpr uint32_t STG_OFF = kStages * STAGE_BYTES;                    // epilogue staging, 1024-byte aligned
     static constexpr uint32_t BAR_OFF = STG_OFF + kEpiWarps * STG_WARP_BYTES;
     static constexpr uint32_t SMEM_BYTES = BAR_OFF + 1024 + 256;
-    static constexpr int kThreads = 128 + 32 * kEpiWarps;
+    static constexpr int kScaleWarps = 2;                          // warps 2 .. 1 + kScaleWarps
+    static constexpr int kFirstEpiWarp = 2 + kScaleWarps;
+    static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     static constexpr uint32_t kTmemSfBase = BN;                                   // accumulator: BN fp32 columns
     static constexpr uint32_t kTmemSfACols = 4 * kKbPerStage;
     static constexpr uint32_t kTmemSfBufCols = kTmemSfACols + 4 * kKbPerStage * kSfbAtoms;
@@ -173,16 +184,25 @@ __device__ __forceinline__ void tile_coords2(int t, int tiles_m, int tiles_n, in
     nb = r / gsz;
 }
 
+// what the gated epilogue (EPI = 1) writes instead of Y
+struct GatedOut {
+    uint8_t *codes;          // [M][F/2] NVFP4 codes of bf16(SiLU(gate) * up)
+    uint8_t *sf;             // their block scales in the MMA's layout
+    float s;                 // static input scale of the layer that reads them
+    int F;                   // features (N = 2F)
+};
+
 // MMA_ONLY (measurement): the same roles and barriers, but no operand or scale loads (the barriers are completed by
 // hand), no scale copies into TMEM and no stores: what is left is the MMA issue sequence on whatever shared memory
 // and TMEM hold, i.e. the tensor-core rate this kernel could reach if nothing else cost time.
-template <bool MMA_ONLY, class C>
+template <bool MMA_ONLY, int EPI, class C>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C::kThreads, C::kMinCtas)
 gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfw,
                        const __grid_constant__ CUtensorMap tmap_y, const PackedHeader *__restrict__ hdr, float act_scale, __nv_bfloat16 *__restrict__ Y,
-                       int64_t ldy, int M, int N, int K, StatusWord *status, int group_m)
+                       int64_t ldy, int M, int N, int K, StatusWord *status, int group_m, GatedOut gated)
 {
+    static_assert(EPI == 0 || C::BN == 256, "the gated epilogue is written for 256-column pair tiles");
     constexpr int BN = C::BN, kStages = C::kStages, kKbPerStage = C::kKbPerStage, kEpiWarps = C::kEpiWarps;
     constexpr int kSfbAtoms = C::kSfbAtoms;
     constexpr uint32_t A_BYTES = C::A_BYTES, B_BYTES = C::B_BYTES, SFA_BYTES = C::SFA_BYTES, SFB_BYTES = C::SFB_BYTES;
@@ -283,19 +303,30 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         }
     } else if (warp == 1) {
         // ------------------------------------------- MMA issuer (leader CTA only)
+        // The tensor pipe takes an MMA of this size every ~130 cycles, so this thread has about 520 cycles per stage
+        // for everything it does, and a barrier probe alone is a round trip to shared memory.  The barriers of the
+        // NEXT stage are therefore probed (without blocking) before the MMAs of this stage are issued and the answer
+        // is read after them; the bounded blocking wait is only the fallback when the ring is not ahead.
         if (rank == 0 && lane == 0) {
             int stage = 0; uint32_t phase = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            bool seen = false;          // barriers of `stage` already seen complete by the look-ahead probe
             const uint32_t a_lo0 = ((smem_base & 0x3FFFFu) >> 4) | (1u << 16);
             for (int t = pair; t < num_tiles && ok; t += npairs) {
                 if (!mbar_wait2(tmem_empty_bar, acc_phase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
                 tc_fence_after();
                 for (int ks = 0; ks < num_ks; ++ks) {
                     // operand tiles of this stage are in smem and its scales are in TMEM
-                    if (!mbar_wait2(full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
-                    if (!mbar_wait2(sf_ready_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                    if (!seen) {
+                        if (!mbar_wait2(full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                        if (!mbar_wait2(sf_ready_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
+                    }
                     tc_fence_after();
+                    const int nstage = (stage + 1 == kStages) ? 0 : stage + 1;
+                    const uint32_t nphase = (stage + 1 == kStages) ? (phase ^ 1u) : phase;
+                    const bool next_full = mbar_test(full_bar(nstage), nphase);
+                    const bool next_sf = mbar_test(sf_ready_bar(nstage), nphase);
                     const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
                     const uint32_t a_lo = a_lo0 + (uint32_t)stage * (STAGE_BYTES >> 4);
                     const uint32_t b_lo = a_lo + (A_BYTES >> 4);
@@ -312,14 +343,16 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         }
                     }
                     mma2_commit_pair(empty_bar(stage));     // stage (smem and TMEM scales) reusable in both CTAs
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    seen = next_full && next_sf;
+                    stage = nstage;
+                    phase = nphase;
                 }
                 if (!ok) break;
                 mma2_commit_pair(tmem_full_bar);
                 acc_phase ^= 1u;
             }
         }
-    } else if (warp == 2 || warp == 3) {
+    } else if (warp < C::kFirstEpiWarp) {
         // ------------------------------- scale copies smem -> TMEM (leader CTA only)
         // One thread can issue only about one copy per 30 ns, and a stage needs 12 of them plus the
         // barrier round trips, which is more than the 0.4 us its MMAs take; so two threads take
@@ -331,7 +364,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             uint32_t step = 0;
             for (int t = pair; t < num_tiles && ok; t += npairs) {
                 for (int ks = 0; ks < num_ks; ++ks, ++step) {
-                    if ((step & 1u) == (uint32_t)(warp - 2)) {
+                    if (step % (uint32_t)C::kScaleWarps == (uint32_t)(warp - 2)) {
                         if (!mbar_wait2(sf_full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
                         tc_fence_after();
                         const int nkb = min(kKbPerStage, katoms - ks * kKbPerStage);
@@ -357,9 +390,9 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 }
             }
         }
-    } else if (warp >= 4) {
+    } else {
         // ------------------------------------------------------------ epilogue
-        const int ew = warp - 4;
+        const int ew = warp - C::kFirstEpiWarp;
         const int wq = warp & 3;                            // TMEM lane quarter this warp may read
         const int half = ew >> 2;                           // which 128 accumulator columns
         const float alpha = __fmul_rn(act_scale, hdr->s);
@@ -410,11 +443,48 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             tmem_ld32(taddr + 96u, v3);
             tmem_ld_wait();
             release_tmem();
-            stage_box(v0, v1, 0);
-            stage_box(v2, v3, 1);
+            if (EPI == 0) {
+                stage_box(v0, v1, 0);
+                stage_box(v2, v3, 1);
+            } else if (!MMA_ONLY) {
+                // columns 0..63 of this warp's slice: gate, 64..127: up, of features f0 .. f0 + 63 of row `row`
+                const int row = row0 + lane;
+                const int f0 = nb * (BN / 2) + half * 64;
+                const float rc6 = __frcp_rn(__fmul_rn(6.0f, gated.s));
+                // G and U as the plain epilogue would have stored them, as packed bf16 pairs
+                uint32_t g2[4][8], u2[4][8];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    g2[i >> 3][i & 7] = pack_bf16x2(__uint_as_float(v0[2 * i]) * alpha, __uint_as_float(v0[2 * i + 1]) * alpha);
+                    g2[2 + (i >> 3)][i & 7] = pack_bf16x2(__uint_as_float(v1[2 * i]) * alpha, __uint_as_float(v1[2 * i + 1]) * alpha);
+                    u2[i >> 3][i & 7] = pack_bf16x2(__uint_as_float(v2[2 * i]) * alpha, __uint_as_float(v2[2 * i + 1]) * alpha);
+                    u2[2 + (i >> 3)][i & 7] = pack_bf16x2(__uint_as_float(v3[2 * i]) * alpha, __uint_as_float(v3[2 * i + 1]) * alpha);
+                }
+                uint32_t cw[8];
+                uint32_t sfw = 0;
+#pragma unroll
+                for (int blk = 0; blk < 4; ++blk) {
+                    uint32_t h[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) h[i] = silu_mul_bf16x2(g2[blk][i], u2[blk][i]);
+                    uint2 c;
+                    sfw |= quant_block_nvfp4_bf16(h, gated.s, rc6, c) << (8 * blk);
+                    cw[2 * blk] = c.x;
+                    cw[2 * blk + 1] = c.y;
+                }
+                if (row < M && f0 < gated.F) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(gated.codes + ((int64_t)row * (gated.F >> 4) + (f0 >> 4)) * 8);
+                    dst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+                    dst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+                    const int rr = row & 127;
+                    const size_t off = ((size_t)(row >> 7) * (size_t)(gated.F >> 6) + (size_t)(f0 >> 6)) * 512 +
+                                       (size_t)((rr & 31) * 16 + (rr >> 5) * 4);
+                    *reinterpret_cast<uint32_t *>(gated.sf + off) = sfw;
+                }
+            }
             acc_phase ^= 1u;
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // all stores of this warp done
+        if (EPI == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this warp done
     }
 
     __syncwarp();
@@ -481,10 +551,12 @@ static cudaError_t launch_pair_cfg(const GemmArgs &a, EncodeTiledFn enc, cudaStr
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false, C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false, 0, C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              C::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<true, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<true, 0, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_nvfp4_pair_kernel<false, 1, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -495,7 +567,11 @@ static cudaError_t launch_pair_cfg(const GemmArgs &a, EncodeTiledFn enc, cudaStr
     if (!make_codes_tmap2(enc, &tmap_w, a.w_codes, a.N, a.K, BN / 2)) return cudaErrorInvalidValue;
     if (!make_sf_tmap(enc, &tmap_sfa, a.a_sf, ((a.M + 127) / 128) * katoms)) return cudaErrorInvalidValue;
     if (!make_sf_tmap(enc, &tmap_sfw, a.w_sf, ((a.N + 255) / 256) * 2 * katoms)) return cudaErrorInvalidValue;
-    if (!make_y_tmap(enc, &tmap_y, a.Y, a.M, a.N, a.ldy)) return cudaErrorInvalidValue;
+    // the gated epilogue stores with plain instructions: its output map is never used, any valid map will do
+    const bool gated = a.gated_codes != nullptr;
+    if (gated) tmap_y = tmap_a;
+    else if (!make_y_tmap(enc, &tmap_y, a.Y, a.M, a.N, a.ldy)) return cudaErrorInvalidValue;
+    GatedOut go = {a.gated_codes, a.gated_sf, a.gated_scale, (int)(a.N / 2)};
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = (int)(((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN));
     int pairs = sms / 2 * C::kMinCtas;
@@ -514,13 +590,17 @@ static cudaError_t launch_pair_cfg(const GemmArgs &a, EncodeTiledFn enc, cudaStr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (a.mma_only)
-        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<true, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+    if (gated)
+        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false, 1, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                                   a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M,
-                                  (int)a.N, (int)a.K, a.status, group_m);
-    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+                                  (int)a.N, (int)a.K, a.status, group_m, go);
+    if (a.mma_only)
+        return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<true, 0, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
+                                  a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M,
+                                  (int)a.N, (int)a.K, a.status, group_m, go);
+    return cudaLaunchKernelEx(&cfg, gemm_nvfp4_pair_kernel<false, 0, C>, tmap_a, tmap_w, tmap_sfa, tmap_sfw, tmap_y, a.hdr,
                               a.act_scale, reinterpret_cast<__nv_bfloat16 *>(a.Y), (int64_t)a.ldy, (int)a.M, (int)a.N,
-                              (int)a.K, a.status, group_m);
+                              (int)a.K, a.status, group_m, go);
 }
 
 }  // namespace

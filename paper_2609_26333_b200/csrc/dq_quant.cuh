@@ -127,4 +127,43 @@ __device__ __forceinline__ uint32_t quant_block_nvfp4_bf16(const uint32_t (&w)[8
     return d8;
 }
 
+// SiLU(g) = g / (1 + exp(-g)) in a fixed fp32 sequence (the same one a CPU evaluation can follow bit for bit):
+//   exp(-g) = 2^t, t = -g log2(e): n = rint(t clamped to +-126), f = fma(g, -L_hi, -n), f = fma(g, -L_lo, f),
+//   p = degree-7 Taylor polynomial of 2^f by fused multiply-adds, e = p * 2^n;  silu = g / (1 + e) by IEEE divide.
+__device__ __forceinline__ float silu_f32(float g)
+{
+    const float L_HI = 1.4426950216293335f, L_LO = 1.925963033500256e-08f;      // log2(e) = L_HI + L_LO
+    const float t = __fmul_rn(g, -L_HI);
+    const float n = rintf(fminf(fmaxf(t, -126.0f), 126.0f));
+    float f = __fmaf_rn(g, -L_HI, -n);
+    f = __fmaf_rn(g, -L_LO, f);
+    f = fminf(fmaxf(f, -1.0f), 1.0f);
+    float p = 1.5252733804059841e-05f;
+    p = __fmaf_rn(p, f, 0.00015403530393381608f);
+    p = __fmaf_rn(p, f, 0.0013333558146428443f);
+    p = __fmaf_rn(p, f, 0.009618129107628477f);
+    p = __fmaf_rn(p, f, 0.05550410866482158f);
+    p = __fmaf_rn(p, f, 0.2402265069591007f);
+    p = __fmaf_rn(p, f, 0.6931471805599453f);
+    p = __fmaf_rn(p, f, 1.0f);
+    const float e = __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
+    return __fdiv_rn(g, __fadd_rn(1.0f, e));
+}
+
+// two floats -> packed bf16 pair, round to nearest even, `lo` in the low half
+__device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// h = bf16( SiLU(g) * u ) on packed bf16 pairs
+__device__ __forceinline__ uint32_t silu_mul_bf16x2(uint32_t g2, uint32_t u2)
+{
+    const float lo = __fmul_rn(silu_f32(__uint_as_float(g2 << 16)), __uint_as_float(u2 << 16));
+    const float hi = __fmul_rn(silu_f32(__uint_as_float(g2 & 0xFFFF0000u)), __uint_as_float(u2 & 0xFFFF0000u));
+    return pack_bf16_rn(lo, hi);
+}
+
 }  // namespace dq

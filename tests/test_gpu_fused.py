@@ -55,6 +55,22 @@ def test_rmsnorm_quantiser_bit_exact(dq, oracle, M, K, kind):
     assert np.array_equal(_np(codes), rc)
 
 
+def test_device_silu_equals_the_cpu_sequence_for_every_bf16_input(dq, oracle):
+    """The gate value reaches SiLU as a bf16 number, so there are 65536 inputs: every finite one through the device
+    routine (branch-free divide inside its range, the plain divide outside) against the oracle's fp32 sequence, bit for
+    bit -- zeros with their sign, denormals, the largest magnitudes."""
+    bits = np.arange(65536, dtype=np.uint32)
+    finite = ((bits >> 7) & 0xFF) != 0xFF
+    bits = bits[finite].astype(np.uint16)
+    g = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(DEV)
+    got = dq.test_silu(g).cpu().numpy().view(np.uint32)
+    _status_ok(dq)
+    gf = (bits.astype(np.uint32) << 16).view(np.float32)
+    ref = np.array([oracle.silu_f32(float(x)) for x in gf], dtype=np.float32).view(np.uint32)
+    bad = np.flatnonzero(got != ref)
+    assert bad.size == 0, f"{bad.size} inputs differ, first g = {gf[bad[0]]!r}: {got[bad[0]]:#x} vs {ref[bad[0]]:#x}"
+
+
 @pytest.mark.parametrize("M,F", [(64, 256), (300, 640), (130, 17408)])
 def test_silu_mul_quantiser_bit_exact(dq, oracle, M, F):
     GU = dq_inputs.gaussian_bf16(M, 2 * F, 2.0, 410 + M)
@@ -109,3 +125,104 @@ def test_prefill_linear_on_fused_stages(dq, oracle):
     # a row stride below 2 K is rejected before anything is launched
     rc = dq.lib().dq_prefill_silu_mul_quantize(w_d.handle, GU.data_ptr(), M, F, float(sa2), ws.data_ptr(), ws.numel(), None)
     assert rc == 3
+
+
+def _workspace_codes_scales(ws: torch.Tensor, M: int, F: int):
+    """Canonical (rows x F/2 codes, rows x F/16 scales) view of an activation workspace: the codes are stored row-major
+    at its start, the scales in 512-byte atoms of 128 rows x 4 blocks (rows r, r+32, r+64, r+96 side by side)."""
+    raw = ws.cpu().numpy()
+    codes = raw[: M * F // 2].reshape(M, F // 2).copy()
+    sf_off = (M * F // 2 + 1023) // 1024 * 1024
+    r = np.arange(M)[:, None]
+    b = np.arange(F // 16)[None, :]
+    off = ((r >> 7) * (F // 64) + (b >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (b & 3)
+    return codes, raw[sf_off + off]
+
+
+def _e2m1_values(codes: np.ndarray) -> np.ndarray:
+    mags = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    lo, hi = codes & 0xF, codes >> 4
+    v = np.empty(codes.shape[:-1] + (codes.shape[-1] * 2,))
+    v[..., 0::2] = np.where(lo & 8, -1.0, 1.0) * mags[lo & 7]
+    v[..., 1::2] = np.where(hi & 8, -1.0, 1.0) * mags[hi & 7]
+    return v
+
+
+def _e4m3_values(b: np.ndarray) -> np.ndarray:
+    e, m = (b >> 3) & 0xF, b & 7
+    return np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7))
+
+
+@pytest.mark.parametrize("M,H,F", [(320, 512, 1024), (100, 256, 128), (700, 1024, 2304)])
+def test_gate_up_gemm_with_gated_epilogue(dq, oracle, M, H, F):
+    """Gate/up GEMM whose epilogue gates and quantises for the down projection (App. C.1): (a) for M > 128 the same bits
+    as the GEMM followed by the fused SiLU*up quantiser; (b) against the oracle end to end -- quantised input, fp64
+    product, bf16, SiLU*up, NVFP4 -- where the only freedom is the summation order of the GEMM, which moves a bf16
+    rounding of G or U now and then and with it, rarely, a code; (c) the down projection on top of it."""
+    Wg = dq_inputs.gaussian_bf16(F, H, 0.05, 430)
+    Wu = dq_inputs.gaussian_bf16(F, H, 0.05, 431)
+    Wd = dq_inputs.gaussian_bf16(H, F, 0.02, 432)
+    A = dq_inputs.gaussian_bf16(M, H, 1.0, 433)
+    order = dq.gate_up_row_order(F)
+    Wgu = torch.cat([Wg, Wu], 0)
+    w_il = dq.pack_weights(Wgu[order].contiguous().to(DEV), formats=dq.FMT_NVFP4)       # interleaved rows
+    w_d = dq.pack_weights(Wd.to(DEV), formats=dq.FMT_NVFP4)
+    sa1 = dq_inputs.static_act_scale(A)
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w_il, M), DEV)
+    ows = dq.alloc_workspace(dq.prefill_workspace_bytes(w_d, M), DEV)
+    ows.fill_(0xA5)
+    dq.prefill_quantize(w_il, A.to(DEV), sa1, ws)
+    # the oracle's route: a fused tensor has one global scale, whatever the order of its rows
+    ref_gu = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(Wgu))
+    ref_d = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(Wd))
+    Yr, Sr = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa1, ref_gu["nvfp4_codes"], ref_gu["nvfp4_scales"], ref_gu["s"])
+    GU_ref = torch.from_numpy(Yr).to(torch.bfloat16)                                     # [gate | up], bf16 as stored
+    h_ref = oracle.silu_mul_bf16(dq_inputs.bf16_to_f32_numpy(GU_ref))
+    sa2 = float(np.abs(h_ref).max()) / 2688.0
+    rc, rs = oracle.quant_nvfp4(h_ref, sa2)
+    dq.prefill_gemm_silu_mul_quantize(w_il, M, sa1, ws, w_d, sa2, ows)
+    _status_ok(dq)
+    codes, scales = _workspace_codes_scales(ows, M, F)
+    # (b) against the oracle
+    code_diff = np.count_nonzero(((codes ^ rc) & 0x0F) != 0) + np.count_nonzero(((codes ^ rc) & 0xF0) != 0)
+    scale_diff = np.count_nonzero(scales != rs)
+    assert code_diff <= 2e-3 * M * F, f"{code_diff} of {M * F} codes differ from the oracle's"
+    assert scale_diff <= 2e-3 * M * F / 16, f"{scale_diff} of {M * F // 16} block scales differ from the oracle's"
+    h_gpu = _e2m1_values(codes) * np.repeat(_e4m3_values(scales), 16, axis=1) * sa2
+    h_orc = _e2m1_values(rc) * np.repeat(_e4m3_values(rs), 16, axis=1) * sa2
+    assert np.linalg.norm(h_gpu - h_orc) <= 5e-3 * np.linalg.norm(h_orc)
+    # (a) the two-call path on the same handle: interleaved columns back to [gate | up], then the fused quantiser
+    if M > 128:
+        GU_il = torch.empty(M, 2 * F, dtype=torch.bfloat16, device=DEV)
+        dq.prefill_gemm(w_il, M, sa1, GU_il, ws)
+        GU = torch.empty_like(GU_il)
+        GU[:, order.to(DEV)] = GU_il
+        check_outputs(GU.float().cpu().numpy().astype(np.float64), Yr, Sr, "gate/up, interleaved rows")
+        ows2 = dq.alloc_workspace(dq.prefill_workspace_bytes(w_d, M), DEV)
+        dq.prefill_silu_mul_quantize(w_d, GU, sa2, ows2)
+        _status_ok(dq)
+        c2, s2 = _workspace_codes_scales(ows2, M, F)
+        assert np.array_equal(codes, c2) and np.array_equal(scales, s2)
+    # (c) the down projection reads what the epilogue wrote
+    Y = torch.empty(M, H, dtype=torch.bfloat16, device=DEV)
+    dq.prefill_gemm(w_d, M, sa2, Y, ows)
+    _status_ok(dq)
+    Yd, Sd = oracle.prefill_linear(h_ref, sa2, ref_d["nvfp4_codes"], ref_d["nvfp4_scales"], ref_d["s"])
+    Yg = Y.float().cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(Yg - Yd) <= 6e-3 * np.linalg.norm(Yd)
+
+
+def test_gate_up_gemm_with_gated_epilogue_arguments(dq):
+    F, H, M = 256, 256, 64
+    w_gu = dq.pack_weights(dq_inputs.gaussian_bf16(2 * F, H, 0.05, 440).to(DEV), formats=dq.FMT_NVFP4)
+    w_d = dq.pack_weights(dq_inputs.gaussian_bf16(H, F, 0.02, 441).to(DEV), formats=dq.FMT_NVFP4)
+    w_bad = dq.pack_weights(dq_inputs.gaussian_bf16(H, 2 * F, 0.02, 442).to(DEV), formats=dq.FMT_NVFP4)
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w_gu, M), DEV)
+    ows = dq.alloc_workspace(dq.prefill_workspace_bytes(w_bad, M), DEV)
+    call = dq.lib().dq_prefill_gemm_silu_mul_quantize
+    assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), w_bad.handle, 1.0, ows.data_ptr(), ows.numel(), None) == 2   # shape
+    assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), w_d.handle, 0.0, ows.data_ptr(), ows.numel(), None) == 1     # scale
+    assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), w_d.handle, 1.0, ows.data_ptr(), 1024, None) == 4            # workspace
+    assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), w_d.handle, 1.0, ws.data_ptr(), ws.numel(), None) == 1       # overlap
+    assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), None, 1.0, ows.data_ptr(), ows.numel(), None) == 1
+    _status_ok(dq)
