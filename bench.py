@@ -324,6 +324,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-b2b", action="store_true", help="skip the back-to-back decode loops (short profiling runs)")
+    ap.add_argument("--no-ffn", action="store_true", help="skip the gated FFN chain (gate/up, SiLU*up, down) measurement")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # asked for N GPUs outside a launcher: start N ranks (one per GPU) of this same command
@@ -540,6 +541,51 @@ def main():
                          "bytes per element of norm + quantiser) that the fused kernels do not make"}
         del GU
 
+    # ---- the gated FFN this matrix belongs to (outside the timed region): fused gate/up projection (2N x K, rows
+    #      interleaved for the gated epilogue), SiLU(gate)*up, down projection (K x N), once with the bf16 gate/up
+    #      matrix written and read back (three calls) and once with the gating and the quantiser in the GEMM's
+    #      epilogue (two calls); the activation quantiser in front is the same in both and is included
+    ffn = None
+    if not args.no_b2b and not args.no_ffn and N % 128 == 0:
+        gen = torch.Generator(device=dev).manual_seed(6)
+        Wgu = (torch.randn(2 * N, K, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        w_gu = dq.pack_weights(Wgu, formats=dq.FMT_NVFP4)
+        del Wgu
+        Wd = (torch.randn(K, N, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        w_dn = dq.pack_weights(Wd, formats=dq.FMT_NVFP4)
+        del Wd
+        ws_in = dq.alloc_workspace(dq.prefill_workspace_bytes(w_gu, M), dev)
+        ws_h = dq.alloc_workspace(dq.prefill_workspace_bytes(w_dn, M), dev)
+        GU = torch.empty(M, 2 * N, dtype=torch.bfloat16, device=dev)
+        Yf = torch.empty(M, K, dtype=torch.bfloat16, device=dev)
+        sh = 1.0 / 2688.0
+
+        def ffn_unfused():
+            dq.prefill_quantize(w_gu, A, sa, ws_in)
+            dq.prefill_gemm(w_gu, M, sa, GU, ws_in)
+            dq.prefill_silu_mul_quantize(w_dn, GU, sh, ws_h)
+            dq.prefill_gemm(w_dn, M, sh, Yf, ws_h)
+
+        def ffn_fused():
+            dq.prefill_quantize(w_gu, A, sa, ws_in)
+            dq.prefill_gemm_silu_mul_quantize(w_gu, M, sa, ws_in, w_dn, sh, ws_h)
+            dq.prefill_gemm(w_dn, M, sh, Yf, ws_h)
+
+        t_un, t_fu = timed(ffn_unfused), timed(ffn_fused)
+        t_g = timed(lambda: dq.prefill_gemm(w_gu, M, sa, GU, ws_in))
+        t_gg = timed(lambda: dq.prefill_gemm_silu_mul_quantize(w_gu, M, sa, ws_in, w_dn, sh, ws_h))
+        t_s = timed(lambda: dq.prefill_silu_mul_quantize(w_dn, GU, sh, ws_h))
+        t_d = timed(lambda: dq.prefill_gemm(w_dn, M, sh, Yf, ws_h))
+        fl = 2.0 * M * (2 * N) * K + 2.0 * M * K * N
+        ffn = {"M": M, "hidden": K, "features": N, "three_call_ms": t_un, "gated_epilogue_ms": t_fu,
+               "three_call_tflops": fl / (t_un * 1e-3) / 1e12, "gated_epilogue_tflops": fl / (t_fu * 1e-3) / 1e12,
+               "gate_up_gemm_ms": t_g, "gate_up_gemm_gated_ms": t_gg, "silu_mul_quantize_ms": t_s, "down_gemm_ms": t_d,
+               "bf16_intermediate_bytes_avoided": 2 * 2 * M * 2 * N}
+        st, det = dq.get_status()
+        if st != 0:
+            raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the FFN chain")
+        del GU, Yf, ws_in, ws_h, w_gu, w_dn
+
     # ---- end to end: pinned host buffers, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -659,6 +705,8 @@ def main():
                                                       "timing": "back-to-back launches replayed from one CUDA graph (test hook)"}
     if fused:
         line["fused_activation_stage"] = fused
+    if ffn:
+        line["gated_ffn"] = ffn
     if e2e:
         line["e2e"] = {"value": world * flops / (e2e_p_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": int(2 * M * K + 2 * B * K), "d2h_bytes_per_step": int(2 * M * N + 2 * B * N),
