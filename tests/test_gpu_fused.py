@@ -226,3 +226,48 @@ def test_gate_up_gemm_with_gated_epilogue_arguments(dq):
     assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), w_d.handle, 1.0, ws.data_ptr(), ws.numel(), None) == 1       # overlap
     assert call(w_gu.handle, M, 1.0, ws.data_ptr(), ws.numel(), None, 1.0, ows.data_ptr(), ows.numel(), None) == 1
     _status_ok(dq)
+
+
+def test_gated_ffn_on_lut3_only_handles_and_from_a_cuda_graph(dq):
+    """The gated chain on handles that store LUT3 only (both projections cast to NVFP4 per call, Sec. 2.3) gives, bit
+    for bit, what handles with the pack-time NVFP4 view give; captured in a CUDA graph and replayed on new activations
+    it gives what the eager calls give."""
+    M, H, F = 384, 512, 768
+    order = dq.gate_up_row_order(F)
+    Wgu = torch.cat([dq_inputs.gaussian_bf16(F, H, 0.05, 450), dq_inputs.gaussian_bf16(F, H, 0.05, 451)], 0)[order].contiguous().to(DEV)
+    Wd = dq_inputs.gaussian_bf16(H, F, 0.02, 452).to(DEV)
+    A = dq_inputs.gaussian_bf16(M, H, 1.0, 453).to(DEV)
+    sa1, sa2 = 5.0 / 2688.0, 2.0 / 2688.0
+    outs = []
+    for fmt in (dq.FMT_LUT3, dq.FMT_NVFP4_FROM_LUT3):
+        w_gu, w_d = dq.pack_weights(Wgu, formats=fmt), dq.pack_weights(Wd, formats=fmt)
+        ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w_gu, M), DEV)
+        ows = dq.alloc_workspace(dq.prefill_workspace_bytes(w_d, M), DEV)
+        ws.fill_(0xFF); ows.fill_(0xFF)
+        Y = torch.empty(M, H, dtype=torch.bfloat16, device=DEV)
+
+        def chain():
+            dq.prefill_quantize(w_gu, A, sa1, ws)
+            dq.prefill_gemm_silu_mul_quantize(w_gu, M, sa1, ws, w_d, sa2, ows)
+            dq.prefill_gemm(w_d, M, sa2, Y, ows)
+
+        chain()
+        _status_ok(dq)
+        outs.append(Y.clone())
+        if fmt == dq.FMT_LUT3:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                chain()
+            A0 = A.clone()
+            A.copy_(dq_inputs.gaussian_bf16(M, H, 1.0, 454).to(DEV))
+            Y.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            got = Y.clone()
+            chain()
+            _status_ok(dq)
+            assert torch.equal(got, Y)
+            assert not torch.equal(got, outs[0])
+            A.copy_(A0)
+    assert torch.equal(outs[0], outs[1])
+    assert float(outs[0].float().abs().max()) > 0.0
