@@ -276,7 +276,43 @@ def run_stack(args):
     torch.cuda.synchronize()
     clocks_loop = sampler2.stop()
     d_loop_ms = l0.elapsed_time(l1) / 10
-    p_ms, d_ms, d_loop_ms = replicas.max_over_ranks([p_ms, d_ms, d_loop_ms], device=dev)
+    # the same prefill pass with every layer's gate/up -> down pair chained through the gated epilogue (the gate/up GEMM
+    # gates and quantises for the down projection; the M x 2F bf16 matrix and the down projection's quantiser pass
+    # are gone); random weights stand for interleaved rows as well as for any other order.  Outside `value`; timed
+    # alternately with the plain pass, because both run under the power cap.
+    ws_h = dq.alloc_workspace(max(dq.prefill_workspace_bytes(w, M) for c, w in stack if c.name.endswith("_down")), dev)
+    sh = 1.0 / 2688.0
+
+    def prefill_pass_gated():
+        for i, (cfg, w) in enumerate(stack):
+            if cfg.name.endswith("_gate_up"):
+                dq.prefill_quantize(w, A[cfg.K], sa[cfg.K], workspace)
+                dq.prefill_gemm_silu_mul_quantize(w, M, sa[cfg.K], workspace, stack[i + 1][1], sh, ws_h)
+            elif cfg.name.endswith("_down"):
+                dq.prefill_gemm(w, M, sh, Y[cfg.N], ws_h)
+            else:
+                dq.prefill_quantize(w, A[cfg.K], sa[cfg.K], workspace)
+                dq.prefill_gemm(w, M, sa[cfg.K], Y[cfg.N], workspace)
+
+    prefill_pass_gated()
+    torch.cuda.synchronize()
+    g_ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    g_ev[0].record()
+    prefill_pass()
+    g_ev[1].record()
+    prefill_pass_gated()
+    g_ev[2].record()
+    prefill_pass()
+    g_ev[3].record()
+    prefill_pass_gated()
+    g_ev[4].record()
+    torch.cuda.synchronize()
+    st, det = dq.get_status()
+    if st != 0:
+        raise RuntimeError(f"device status {dq.status_string(st)} (detail {det}) after the gated prefill pass")
+    pg_plain = 0.5 * (g_ev[0].elapsed_time(g_ev[1]) + g_ev[2].elapsed_time(g_ev[3]))
+    pg_gated = 0.5 * (g_ev[1].elapsed_time(g_ev[2]) + g_ev[3].elapsed_time(g_ev[4]))
+    p_ms, d_ms, d_loop_ms, pg_plain, pg_gated = replicas.max_over_ranks([p_ms, d_ms, d_loop_ms, pg_plain, pg_gated], device=dev)
     weights = float(sum(c.N * c.K for c, _ in stack))
     flops = 2.0 * M * weights
     dec_bytes = 0.4375 * weights + sum(2.0 * B * (c.K + c.N) + 4 for c, _ in stack)
@@ -292,7 +328,9 @@ def run_stack(args):
                    "l2": f"inputs larger than L2: packed stack {sum(w.packed.numel() for _, w in stack) / 1e9:.1f} GB",
                    "step": "prefill pass (quantise + GEMM per matrix) + decode token step (one CUDA graph)"},
         "clocks": clocks, "gpu_launches": steps * len(stack) * (2 + passes),
-        "prefill": {"ms": p_ms, "linear_tflops_per_gpu": tflops / world},
+        "prefill": {"ms": p_ms, "linear_tflops_per_gpu": tflops / world,
+                    "gated_ffn_pass_ms": pg_gated, "plain_pass_beside_it_ms": pg_plain,
+                    "gated_ffn_pass_tflops_per_gpu": flops / (pg_gated * 1e-3) / 1e12},
         "decode": {"ms": d_ms, "value": gbs, "unit": "GB/s", "batch": B, "frac_of_measured_hbm": gbs / world / peaks["hbm_gbs"],
                    "token_loop_ms": d_loop_ms, "token_loop_gbs": dec_bytes / (d_loop_ms * 1e-3) / 1e9,
                    "token_loop_frac_of_measured_hbm": dec_bytes / (d_loop_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
