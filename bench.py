@@ -468,6 +468,8 @@ def main():
         step(args.warmup + i, evs[i])
     t_end.record()
     torch.cuda.synchronize()
+    # the last GEMM launch of the timed region as its own first CTA saw it: SM cycles and global-timer nanoseconds
+    gemm_cycles, gemm_ns = dq.bench_gemm_clocks() if M > 128 else (0, 0)
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
@@ -674,6 +676,15 @@ def main():
     burst = total_ms < 1000.0
     fp4_peak = 4.0 * (peaks["bf16_burst"] if burst else peaks["bf16_sustained"])
     sm_mhz = clocks.get("sm_mhz")
+    in_kernel = None
+    if gemm_cycles and gemm_ns:
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        per_clk = 2.0 * M * N * K / (gemm_cycles * sms)
+        in_kernel = {"sm_cycles": gemm_cycles, "us": gemm_ns / 1e3, "sm_mhz": gemm_cycles / gemm_ns * 1e3,
+                     "flop_per_clk_per_sm": per_clk, "frac_of_tensor_pipe_per_clock": per_clk / 32768.0,
+                     "note": "last GEMM launch of the timed region, clock64 and globaltimer on its first CTA's SM; 32768 "
+                             "FLOP per clock and SM = one 128x256x64 FP4 MMA per 128 clocks, the rate the MMA issue "
+                             "sequence reaches between accumulator hand-offs"}
 
     line = {
         "metric": METRIC, "value": prefill_tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -708,7 +719,8 @@ def main():
                      "frac_of_nominal_fp4": gemm_tflops / NOMINAL_FP4_TFLOPS,
                      "fp4_probe_tflops": fp4_probe_tflops,
                      "frac_of_probe": gemm_tflops / fp4_probe_tflops if fp4_probe_tflops else None,
-                     "gemm_ms_x_sm_mhz": g_ms * sm_mhz if sm_mhz else None},
+                     "gemm_ms_x_sm_mhz": g_ms * sm_mhz if sm_mhz else None,
+                     "in_kernel": in_kernel},
         "roofline_decode": {"kernel": "gemv_lut_kernel<3>", "bound": "hbm", "achieved": decode_gbs,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": decode_gbs / peaks["hbm_gbs"],
                             "traffic": NCU_TRAFFIC_BYTES.get(("gemv", cfg.name)) if B == 1 else None,

@@ -326,6 +326,15 @@ int dq_silu_mul_quantize_activations(const void *GU_dev, int64_t M, int64_t F, i
                                      void *stream);
 
 /*
+ * Measurement hook: how long the last CTA-pair GEMM launch on the current device (dq_prefill_gemm with M > 128,
+ * dq_prefill_gemm_silu_mul_quantize, dq_bench_gemm_mma_only) ran on the SM of its first CTA, in SM clock cycles
+ * (clock64) and in nanoseconds of the global timer; their ratio is the SM clock under that load, which on a
+ * power-capped part is lower than what a management query reports between launches.  Synchronises `stream`.
+ * Both values are 0 before the first such launch.
+ */
+int dq_bench_gemm_clocks(void *stream, unsigned long long *sm_cycles_host, unsigned long long *ns_host);
+
+/*
  * Test hook: out[i] = SiLU(g[i]) in fp32 exactly as the gated quantisers evaluate it (dq_prefill_silu_mul_quantize,
  * dq_prefill_gemm_silu_mul_quantize; App. C.1 fused activation processing), for n bf16 values on the device.  There
  * are only 65536 inputs, so a test can compare the fixed fp32 sequence with a CPU evaluation for every one of them.

@@ -22,7 +22,7 @@ SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights
            "dq_prefill_workspace_bytes", "dq_prefill_linear", "dq_prefill_quantize", "dq_prefill_gemm",
            "dq_prefill_linear_static",
            "dq_decode_linear", "dq_decode_linear_nvfp4", "dq_decode_linear_lut2", "dq_test_decode_linear",
-           "dq_bench_gemm_mma_only", "dq_bench_stream_read",
+           "dq_bench_gemm_mma_only", "dq_bench_stream_read", "dq_bench_gemm_clocks",
            "dq_prefill_rmsnorm_quantize", "dq_prefill_silu_mul_quantize", "dq_prefill_gemm_silu_mul_quantize",
            "dq_rmsnorm_quantize_activations",
            "dq_silu_mul_quantize_activations", "dq_test_silu", "dq_export_canonical", "dq_import_canonical",
@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
         L.dq_prefill_rmsnorm_quantize.argtypes = [vp, vp, i64, i64, vp, C.c_float, C.c_float, vp, sz, vp]
         L.dq_prefill_silu_mul_quantize.restype = C.c_int
         L.dq_prefill_silu_mul_quantize.argtypes = [vp, vp, i64, i64, C.c_float, vp, sz, vp]
+        L.dq_bench_gemm_clocks.restype = C.c_int
+        L.dq_bench_gemm_clocks.argtypes = [vp, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong)]
         L.dq_test_silu.restype = C.c_int
         L.dq_test_silu.argtypes = [vp, i64, vp, vp]
         L.dq_prefill_gemm_silu_mul_quantize.restype = C.c_int
@@ -384,6 +386,13 @@ def test_decode_linear(w: DQWeights, fmt: int, X: torch.Tensor, out: torch.Tenso
 
 test_decode_linear.__test__ = False      # not a pytest test
 test_silu.__test__ = False
+
+
+def bench_gemm_clocks(stream=None):
+    """dq_bench_gemm_clocks: (SM clock cycles, nanoseconds) the last CTA-pair GEMM launch took on its first CTA's SM."""
+    cyc, ns = C.c_ulonglong(0), C.c_ulonglong(0)
+    _check(lib().dq_bench_gemm_clocks(_stream_ptr(stream), C.byref(cyc), C.byref(ns)), "dq_bench_gemm_clocks")
+    return int(cyc.value), int(ns.value)
 
 
 def bench_gemm_mma_only(w: DQWeights, M: int, out: torch.Tensor, workspace: torch.Tensor, stream=None):

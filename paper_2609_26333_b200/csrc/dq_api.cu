@@ -701,12 +701,26 @@ int dq_get_status(void *stream, int *status_host, int *detail_host)
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     dq::StatusWord *sw = status_word_ptr();
     if (!sw) return DQ_ERR_CUDA;
-    dq::StatusWord h;
-    if (cudaMemcpyAsync(&h, sw, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DQ_ERR_CUDA;
+    int h[2] = {0, 0};                                     // status and detail: the first two words
+    if (cudaMemcpyAsync(h, sw, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaMemsetAsync(sw, 0, sizeof(h), s) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return DQ_ERR_CUDA;
-    *status_host = h.status;
-    if (detail_host) *detail_host = h.detail;
+    *status_host = h[0];
+    if (detail_host) *detail_host = h[1];
+    return DQ_OK;
+}
+
+int dq_bench_gemm_clocks(void *stream, unsigned long long *sm_cycles_host, unsigned long long *ns_host)
+{
+    if (!sm_cycles_host || !ns_host) return DQ_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    dq::StatusWord *sw = status_word_ptr();
+    if (!sw) return DQ_ERR_CUDA;
+    dq::StatusWord h;
+    if (cudaMemcpyAsync(&h, sw, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return DQ_ERR_CUDA;
+    *sm_cycles_host = h.gemm_cycles;
+    *ns_host = h.gemm_ns;
     return DQ_OK;
 }
 

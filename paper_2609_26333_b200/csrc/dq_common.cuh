@@ -158,8 +158,9 @@ __host__ __device__ inline size_t sf_swizzled_offset(int64_t r, int64_t b, int64
     return (size_t)atom * 512 + (size_t)(rr % 32) * 16 + (size_t)(rr / 32) * 4 + (size_t)(b % 4);
 }
 
-// Device status word: [0] = dq_status, [1] = detail.
-struct StatusWord { int status; int detail; };
+// Device status word: [0] = dq_status, [1] = detail; then, for measurement, what the last pair-GEMM launch took on the
+// SM of its first CTA: SM clock cycles and nanoseconds of the global timer from the CTA's start to its end.
+struct StatusWord { int status; int detail; unsigned long long gemm_cycles; unsigned long long gemm_ns; };
 
 bool handle_on_current_device(const dq_weights *w);      // defined beside the handle (dq_api.cu)
 

@@ -250,6 +250,13 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     // before that kernel has completed.  A dependent kernel may start its own set-up from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // measurement: the SM clock this launch really runs at (the clock a management query reports between launches is
+    // not the clock under this load) -- cycles and global-timer nanoseconds of the first CTA, left in the status word
+    long long clk0 = 0, ns0 = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        clk0 = clock64();
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns0));
+    }
 
     const int tiles_m = (M + 2 * BM - 1) / (2 * BM);
     const int tiles_n = (N + BN - 1) / BN;
@@ -490,6 +497,12 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     __syncwarp();
     tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        long long ns1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+        status->gemm_cycles = (unsigned long long)(clock64() - clk0);
+        status->gemm_ns = (unsigned long long)(ns1 - ns0);
+    }
     cluster_sync_all();            // nobody leaves while the partner may still signal its barriers
     if (*abort_flag) {
         for (int i = 0; i < 200; ++i) __nanosleep(1000);       // let copies in flight land

@@ -700,3 +700,28 @@ def test_decode_wide_batch_kernel_parity(dq, oracle, N, K, seed, B):
     _status_ok(dq)
     Yr, S = oracle.decode_linear_lut2(Xf, planes2, scales2, s2)
     check_outputs(_f64(out[:, :N]), Yr, S, f"wide lut2 decode {B}x{N}x{K}")
+
+
+def test_measurement_hooks_leave_results_alone(dq, oracle):
+    """The measurement hooks (MMA issue sequence alone, streaming read, in-kernel clocks of the last pair GEMM) run, return
+    sane values and do not disturb a following prefill: its output is the one from before, bit for bit."""
+    M, N, K = 512, 1024, 1024
+    W, _ = _layer(oracle, N, K, 90)
+    w = dq.pack_weights(W.to(DEV), formats=dq.FMT_NVFP4)
+    A = dq_inputs.gaussian_bf16(M, K, 1.0, 91).to(DEV)
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w, M), DEV)
+    sa = 4.0 / 2688.0
+    Y0 = dq.prefill_linear(w, A, sa, workspace=ws)
+    cycles, ns = dq.bench_gemm_clocks()
+    assert cycles > 0 and ns > 0
+    assert 500.0 < cycles / ns * 1e3 < 2500.0                  # an SM clock in MHz
+    scratch = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    dq.bench_gemm_mma_only(w, M, scratch, ws)
+    c2, n2 = dq.bench_gemm_clocks()
+    assert c2 > 0 and n2 > 0 and (c2, n2) != (cycles, ns)
+    out = torch.zeros(8, dtype=torch.uint8, device=DEV)
+    dq.bench_stream_read(w.packed[: w.packed.numel() // 16 * 16], out)
+    _status_ok(dq)
+    assert torch.equal(dq.prefill_linear(w, A, sa, workspace=ws), Y0)
+    with pytest.raises(dq.DQError):
+        dq.bench_gemm_mma_only(w, 64, scratch, ws)             # the measurement mode exists for M > 128 only
