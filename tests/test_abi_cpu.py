@@ -92,3 +92,33 @@ def test_binding_fails_loudly_without_library(dq, tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "missing.so")
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_gate_up_row_order_is_the_documented_interleave(dq):
+    """Row 256 t + 128 h + 64 p + j of the interleaved gate/up matrix is gate (p = 0) or up (p = 1) of feature
+    128 t + 64 h + j: a permutation of the 2F rows of [gate; up] in which every 256-row tile holds both halves of the
+    same 128 features, each 128-column half of a tile gate and up of the same 64."""
+    import torch
+    F = 384
+    order = dq.gate_up_row_order(F)
+    assert sorted(order.tolist()) == list(range(2 * F))
+    for r in (0, 63, 64, 127, 128, 191, 192, 255, 256, 700):
+        t, h, p, j = r // 256, (r // 128) % 2, (r // 64) % 2, r % 64
+        assert int(order[r]) == p * F + 128 * t + 64 * h + j
+    for tile in range(2 * F // 256):
+        rows = order[256 * tile: 256 * (tile + 1)]
+        feats = rows % F
+        assert sorted(set(feats.tolist())) == list(range(128 * tile, 128 * (tile + 1)))
+        for half in range(2):
+            g, u = rows[128 * half: 128 * half + 64], rows[128 * half + 64: 128 * half + 128]
+            assert torch.all(g < F) and torch.all(u >= F) and torch.equal(g, u - F)
+    with pytest.raises(AssertionError):
+        dq.gate_up_row_order(200)
+
+
+def test_gated_gemm_entry_point_rejects_bad_arguments_without_a_device(dq):
+    L = dq.lib()
+    assert L.dq_prefill_gemm_silu_mul_quantize(None, 1, C.c_float(1.0), None, 0, None, C.c_float(1.0), None, 0, None) == 1
+    cyc, ns = C.c_ulonglong(0), C.c_ulonglong(0)
+    assert L.dq_bench_gemm_clocks(None, None, C.byref(ns)) == 1
+    assert L.dq_test_silu(None, 0, None, None) == 1
