@@ -158,7 +158,7 @@ def test_gate_up_gemm_with_gated_epilogue(dq, oracle, M, H, F):
     """Gate/up GEMM whose epilogue gates and quantises for the down projection (App. C.1): (a) for M > 128 the same bits
     as the GEMM followed by the fused SiLU*up quantiser; (b) against the oracle end to end -- quantised input, fp64
     product, bf16, SiLU*up, NVFP4 -- where the only freedom is the summation order of the GEMM, which moves a bf16
-    rounding of G or U now and then and with it, rarely, a code; (c) the down projection on top of it."""
+    rounding of G or U now and then and with it, rarely, a code (measured: at most 3 codes in a million, no scale); (c) the down projection on top of it."""
     Wg = dq_inputs.gaussian_bf16(F, H, 0.05, 430)
     Wu = dq_inputs.gaussian_bf16(F, H, 0.05, 431)
     Wd = dq_inputs.gaussian_bf16(H, F, 0.02, 432)
@@ -186,11 +186,11 @@ def test_gate_up_gemm_with_gated_epilogue(dq, oracle, M, H, F):
     # (b) against the oracle
     code_diff = np.count_nonzero(((codes ^ rc) & 0x0F) != 0) + np.count_nonzero(((codes ^ rc) & 0xF0) != 0)
     scale_diff = np.count_nonzero(scales != rs)
-    assert code_diff <= 2e-3 * M * F, f"{code_diff} of {M * F} codes differ from the oracle's"
-    assert scale_diff <= 2e-3 * M * F / 16, f"{scale_diff} of {M * F // 16} block scales differ from the oracle's"
+    assert code_diff <= max(2, 1e-4 * M * F), f"{code_diff} of {M * F} codes differ from the oracle's"
+    assert scale_diff <= max(1, 1e-4 * M * F / 16), f"{scale_diff} of {M * F // 16} block scales differ from the oracle's"
     h_gpu = _e2m1_values(codes) * np.repeat(_e4m3_values(scales), 16, axis=1) * sa2
     h_orc = _e2m1_values(rc) * np.repeat(_e4m3_values(rs), 16, axis=1) * sa2
-    assert np.linalg.norm(h_gpu - h_orc) <= 5e-3 * np.linalg.norm(h_orc)
+    assert np.linalg.norm(h_gpu - h_orc) <= 1e-3 * np.linalg.norm(h_orc)
     # (a) the two-call path on the same handle: interleaved columns back to [gate | up], then the fused quantiser
     if M > 128:
         GU_il = torch.empty(M, 2 * F, dtype=torch.bfloat16, device=DEV)
@@ -209,7 +209,7 @@ def test_gate_up_gemm_with_gated_epilogue(dq, oracle, M, H, F):
     _status_ok(dq)
     Yd, Sd = oracle.prefill_linear(h_ref, sa2, ref_d["nvfp4_codes"], ref_d["nvfp4_scales"], ref_d["s"])
     Yg = Y.float().cpu().numpy().astype(np.float64)
-    assert np.linalg.norm(Yg - Yd) <= 6e-3 * np.linalg.norm(Yd)
+    assert np.linalg.norm(Yg - Yd) <= 2.5e-3 * np.linalg.norm(Yd)          # the bf16 rounding of Y alone is 1.7e-3
 
 
 def test_gate_up_gemm_with_gated_epilogue_arguments(dq):
