@@ -90,3 +90,60 @@ def test_c4_stack_layer_shapes(dq, oracle, which):
     """The matrices of one layer of the 27B-class stack (fused q/k/v, o, fused gate/up, down) at
     4096 prefill tokens and decode batches 1..64; the other 63 layers repeat these shapes."""
     _run_config(dq, oracle, dq_inputs.c4_fused_layer(layer=3)[which], full_rows=False, layer=3)
+
+
+def test_c3_gated_ffn_sampled(dq, oracle):
+    """The gated FFN of the bench line (`gated_ffn`: M = 8192, gate/up 34816 x 5120 with interleaved rows, down
+    5120 x 17408).  Codes and scales the gated epilogue writes: bit for bit the two-call path's, in full; against the
+    oracle (quantised operands, fp64 product, bf16, SiLU*up, NVFP4) on sampled rows, where the GEMM's summation order may
+    move one code in ten thousand; the down projection on those rows against the oracle's product."""
+    from test_gpu_fused import _workspace_codes_scales
+    up_cfg = dq_inputs.LayerConfig("c3_up27b", N=17408, K=5120, M=8192, cfg_id=3, matrix_id=2)
+    gate_cfg, down_cfg = dq_inputs.CONFIGS["c3_gate_up27b"], dq_inputs.CONFIGS["c3_down27b"]
+    M, F, H = gate_cfg.M, gate_cfg.N, gate_cfg.K
+    Wgu = torch.cat([dq_inputs.make_weight(gate_cfg), dq_inputs.make_weight(up_cfg)], 0)         # [gate; up], one tensor
+    Wd = dq_inputs.make_weight(down_cfg)
+    A = dq_inputs.make_activations(gate_cfg, M)
+    sa1 = dq_inputs.static_act_scale(A)
+    order = dq.gate_up_row_order(F)
+    w_gu = dq.pack_weights(Wgu[order].contiguous().to(DEV), formats=dq.FMT_NVFP4)
+    w_d = dq.pack_weights(Wd.to(DEV), formats=dq.FMT_NVFP4)
+    ws = dq.alloc_workspace(dq.prefill_workspace_bytes(w_gu, M), DEV)
+    ows = dq.alloc_workspace(dq.prefill_workspace_bytes(w_d, M), DEV)
+    ows2 = dq.alloc_workspace(dq.prefill_workspace_bytes(w_d, M), DEV)
+    dq.prefill_quantize(w_gu, A.to(DEV), sa1, ws)
+    # the static scale of the down projection's input: from a calibration pass of the two-call path
+    GU_il = torch.empty(M, 2 * F, dtype=torch.bfloat16, device=DEV)
+    dq.prefill_gemm(w_gu, M, sa1, GU_il, ws)
+    GU = torch.empty_like(GU_il)
+    GU[:, order.to(DEV)] = GU_il
+    del GU_il
+    h_abs = (torch.nn.functional.silu(GU[:, :F].float()) * GU[:, F:].float()).abs().max()
+    sa2 = float(h_abs) / 2688.0
+    dq.prefill_gemm_silu_mul_quantize(w_gu, M, sa1, ws, w_d, sa2, ows)
+    dq.prefill_silu_mul_quantize(w_d, GU, sa2, ows2)
+    Y = torch.empty(M, H, dtype=torch.bfloat16, device=DEV)
+    dq.prefill_gemm(w_d, M, sa2, Y, ows)
+    torch.cuda.synchronize()
+    st, det = dq.get_status()
+    assert st == 0, (st, det)
+    del GU
+    codes, scales = _workspace_codes_scales(ows, M, F)
+    c2, s2 = _workspace_codes_scales(ows2, M, F)
+    assert np.array_equal(codes, c2) and np.array_equal(scales, s2)
+    # the oracle on sampled rows
+    rng = np.random.default_rng(321)
+    rows = np.unique(np.concatenate([rng.choice(M, 24, replace=False), np.array([0, 127, 128, 255, 256, M - 129, M - 128, M - 1])]))
+    ref_gu = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(Wgu))
+    Yr, _ = oracle.prefill_linear(dq_inputs.bf16_to_f32_numpy(A), sa1, ref_gu["nvfp4_codes"], ref_gu["nvfp4_scales"], ref_gu["s"],
+                                  rows=rows)
+    h_ref = oracle.silu_mul_bf16(dq_inputs.bf16_to_f32_numpy(torch.from_numpy(Yr).to(torch.bfloat16)))
+    rc, rs = oracle.quant_nvfp4(h_ref, sa2)
+    code_diff = np.count_nonzero(((codes[rows] ^ rc) & 0x0F) != 0) + np.count_nonzero(((codes[rows] ^ rc) & 0xF0) != 0)
+    scale_diff = np.count_nonzero(scales[rows] != rs)
+    assert code_diff <= 1e-4 * rows.size * F, f"{code_diff} of {rows.size * F} codes differ from the oracle's"
+    assert scale_diff <= 1e-4 * rows.size * F / 16, f"{scale_diff} block scales differ from the oracle's"
+    ref_d = oracle.pack_weights(dq_inputs.bf16_to_f32_numpy(Wd))
+    Yd, _ = oracle.prefill_linear(h_ref, sa2, ref_d["nvfp4_codes"], ref_d["nvfp4_scales"], ref_d["s"])
+    Yg = _f64(Y[torch.from_numpy(rows).to(DEV)])
+    assert np.linalg.norm(Yg - Yd) <= 2.5e-3 * np.linalg.norm(Yd)
