@@ -220,8 +220,8 @@ int dq_prefill_linear_static(const dq_weights *w, const void *A_dev, int64_t M, 
  * fp32 rounding errors of sum_k |x w| plus the bf16 rounding of the result, for any activation
  * pattern.  An activation more than 2^28 times smaller in magnitude than the largest activation
  * it shares a power-of-two scale with loses low bits or reads as zero: that is the largest of the
- * same pass (up to eight rows of X), or, for batches above 8 on matrices of more than about 14000
- * rows, of the same 1024-element slice of K of the same pass (up to 32 rows of X).
+ * same pass (up to eight rows of X), or, for batches above 8 on matrices of 8192 rows and more (4096 and
+ * more from batch 16 on), of the same 1024-element slice of K of the same pass (up to 32 rows of X).
  * X_dev: B x K bf16, row stride ldx; Y_dev: B x N bf16, row stride ldy.
  */
 int dq_decode_linear(const dq_weights *w, const void *X_dev, int64_t B, int64_t ldx,
@@ -370,9 +370,9 @@ int dq_weights_shape(const dq_weights *w, int64_t *N_host, int64_t *K_host, unsi
  *           arithmetic; measured slower than the default kernel, it is kept for comparison and is
  *           not what dq_decode_linear launches.  The three split arguments do not apply to it.
  *           variant 4 runs the kernel that dq_decode_linear takes for batches above 8 on matrices
- *           of more than about 14000 rows (up to 32 columns in one pass over the weights, 16-row
+ *           of 8192 rows and more (up to 32 columns in one pass over the weights, 16-row
  *           tiles, K walked in slices of 1024 with a power-of-two activation scale per slice) on
- *           any shape and batch.
+ *           any shape and batch; groups_per_cta (1..9) then sets its warps per CTA.
  *   format  DQ_FMT_NVFP4 / DQ_FMT_NVFP4_FROM_LUT3: the NVFP4A16 decode; variant 0 = the tensor-core
  *           kernel dq_decode_linear_nvfp4 runs, 1 = the CUDA-core kernel kept for comparison.
  * Other arguments as dq_decode_linear.

@@ -863,14 +863,14 @@ cudaError_t launch_wide(const GemvArgs &a, int sms, cudaStream_t stream)
 {
     const int64_t ntiles = a.N / 16;
     const uint32_t stage = 4u * (uint32_t)lut_atom_bytes(a.bits);
-    // Warps per CTA (each owns one 16-row tile per round): as few tiles on the busiest SM as the rounds allow, among
-    // the counts whose rings fit beside 32 columns of a slice; of equals the larger.
-    int G = 4;
-    int64_t best = -1;
-    for (int cand = 4; cand <= 9; ++cand) {
-        const int64_t busiest = ((ntiles + (int64_t)sms * cand - 1) / ((int64_t)sms * cand)) * cand;
-        if (best < 0 || busiest <= best) { best = busiest; G = cand; }
-    }
+    // Warps per CTA (each owns one 16-row tile per round): eight, two per scheduler.  A round takes about as long with
+    // four warps as with eight (each warp is bound by the latency of its own instruction chain, and every CTA pays for
+    // staging the slice whatever its size), nine put a third warp on one scheduler and that one sets the pace; so the
+    // rounds are what counts, and fewer, fuller CTAs beat more, emptier ones even when SMs stay idle (measured on
+    // ten shapes from 1024 to 34816 rows: 34816 x 5120 at batch 32, 85 us with 8 warps, 171 us with 5 warps and one
+    // tile less on the busiest SM).
+    int G = ntiles < 8 ? (int)ntiles : 8;
+    if (a.force_G >= 1 && a.force_G <= 9) G = a.force_G;       // test hook
     WidePlan L;
     L.bar_off = 1024;
     L.sbuf_off = 2048;
@@ -1022,7 +1022,9 @@ cudaError_t launch_gemv_lut(const GemvArgs &a, cudaStream_t stream)
         return launch_gemv_lut_tc(a, wgs, stream);
     }
     // batches above 8 on enough rows to give every SM several 16-row tiles: the kernel that walks K slice by slice
-    if ((a.kernel == 3 || (a.kernel == 0 && a.force_P == 0 && B > 8 && (int64_t)N / 16 > (int64_t)sms * 6)))
+    // Batches above 8: one slice-by-slice pass over the weights per 32 columns instead of one pass per 8 columns, where
+    // that is faster (measured: from 8192 rows on, and from 4096 rows on for 16 columns and more)
+    if ((a.kernel == 3 || (a.kernel == 0 && a.force_P == 0 && B > 8 && (N >= 8192 || (B >= 16 && N >= 4096)))))
         return launch_wide(a, sms, stream);
     const int want_cols = B;                    // the split decides how many of them one pass takes
     Split sp = choose_split(a.bits, N, K, sms, want_cols);
