@@ -297,13 +297,22 @@ int dq_export_canonical(const dq_weights *w, unsigned format, void *codes_dev, v
  * need lut3_planes_dev / lut3_scales_dev (unused pointers may be NULL); global_scale is the tensor
  * scale s (finite, > 0), shared by both encodings.  packed_dev / packed_bytes / ownership as in
  * dq_pack_weights.  No value check is made on the codes: every bit pattern decodes to something.
- * DQ_FMT_LUT2 cannot be imported (DQ_ERR_INVALID_ARG): it is packed from master weights only.
+ * DQ_FMT_LUT2 is imported on its own with dq_import_canonical_lut2 (passing it here: DQ_ERR_INVALID_ARG).
  */
 int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp4_codes_dev,
                         const void *nvfp4_scales_dev, const void *lut3_planes_dev,
                         const void *lut3_scales_dev, float global_scale,
                         const uint16_t *lut3_codebook_f16_host, void *packed_dev, size_t packed_bytes,
                         void *stream, dq_weights **out_host);
+
+/*
+ * A DQ_FMT_LUT2 handle from canonical LUT2 encodings (planes uint32[N][2][K/32], scales uint8[N][K/16] signed E4M3,
+ * device pointers; App. A.3 "LUT formats", the 4-level grid) and the tensor scale.  The result decodes with
+ * dq_decode_linear_lut2.  Other arguments, ownership and status codes as dq_import_canonical.
+ */
+int dq_import_canonical_lut2(int64_t N, int64_t K, const void *lut2_planes_dev, const void *lut2_scales_dev,
+                             float global_scale, void *packed_dev, size_t packed_bytes, void *stream,
+                             dq_weights **out_host);
 
 /*
  * The activation quantiser of dq_prefill_linear on its own (App. A.3 "NVFP4",

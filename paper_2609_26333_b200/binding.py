@@ -26,6 +26,7 @@ SYMBOLS = ("dq_version", "dq_status_string", "dq_packed_bytes", "dq_pack_weights
            "dq_prefill_rmsnorm_quantize", "dq_prefill_silu_mul_quantize", "dq_prefill_gemm_silu_mul_quantize",
            "dq_rmsnorm_quantize_activations",
            "dq_silu_mul_quantize_activations", "dq_test_silu", "dq_export_canonical", "dq_import_canonical",
+           "dq_import_canonical_lut2",
            "dq_quantize_activations", "dq_get_status", "dq_weights_shape",
            "dq_prefill_host_staging_bytes", "dq_prefill_linear_host", "dq_decode_linear_host")
 
@@ -105,6 +106,8 @@ def lib() -> C.CDLL:
         L.dq_import_canonical.restype = C.c_int
         L.dq_import_canonical.argtypes = [C.c_int64, C.c_int64, C.c_uint, vp, vp, vp, vp, C.c_float,
                                           C.POINTER(C.c_uint16), vp, C.c_size_t, vp, C.POINTER(vp)]
+        L.dq_import_canonical_lut2.restype = C.c_int
+        L.dq_import_canonical_lut2.argtypes = [C.c_int64, C.c_int64, vp, vp, C.c_float, vp, C.c_size_t, vp, C.POINTER(vp)]
         L.dq_export_canonical.restype = C.c_int
         L.dq_export_canonical.argtypes = [vp, C.c_uint, vp, vp, vp, vp]
         L.dq_quantize_activations.restype = C.c_int
@@ -209,6 +212,22 @@ def import_canonical(N: int, K: int, formats: int, global_scale: float, nvfp4=No
     if formats & FMT_NVFP4_FROM_LUT3:
         formats |= FMT_LUT3
     return DQWeights(out.value, packed, N, K, formats)
+
+
+def import_canonical_lut2(N: int, K: int, global_scale: float, planes: torch.Tensor, scales: torch.Tensor,
+                          stream=None) -> DQWeights:
+    """dq_import_canonical_lut2: a LUT2 handle from canonical bit-planes (N, 2, K/32) and scales (N, K/16)."""
+    assert planes.is_cuda and planes.is_contiguous() and tuple(planes.shape) == (N, 2, K // 32)
+    assert scales.is_cuda and scales.is_contiguous() and tuple(scales.shape) == (N, K // 16)
+    nbytes = packed_bytes(N, K, FMT_LUT2)
+    packed = torch.empty(nbytes + 1024, dtype=torch.uint8, device=planes.device)
+    off = (-packed.data_ptr()) % 1024
+    view = packed[off:off + nbytes]
+    out = C.c_void_p(0)
+    _check(lib().dq_import_canonical_lut2(N, K, planes.data_ptr(), scales.data_ptr(), float(global_scale),
+                                          view.data_ptr(), nbytes, _stream_ptr(stream), C.byref(out)),
+           "dq_import_canonical_lut2")
+    return DQWeights(out.value, packed, N, K, FMT_LUT2)
 
 
 def prefill_workspace_bytes(w: DQWeights, M: int) -> int:

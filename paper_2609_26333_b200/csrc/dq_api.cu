@@ -293,6 +293,46 @@ int dq_import_canonical(int64_t N, int64_t K, unsigned formats, const void *nvfp
     return DQ_OK;
 }
 
+int dq_import_canonical_lut2(int64_t N, int64_t K, const void *lut2_planes_dev, const void *lut2_scales_dev,
+                             float global_scale, void *packed_dev, size_t packed_bytes, void *stream,
+                             dq_weights **out_host)
+{
+    if (!packed_dev || !out_host || !lut2_planes_dev || !lut2_scales_dev) return DQ_ERR_INVALID_ARG;
+    const unsigned formats = DQ_FMT_LUT2;
+    int st = check_shape(N, K, formats);
+    if (st != DQ_OK) return st;
+    if (!(global_scale > 0.0f) || !std::isfinite(global_scale)) return DQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 1024) || !aligned(lut2_planes_dev, 4)) return DQ_ERR_ALIGN;
+    uint16_t cb[8];
+    default_codebook(cb);                                  // header field of the LUT3 grid; the LUT2 grid is fixed
+    st = check_arch();
+    if (st != DQ_OK) return st;
+    const dq::PackedLayout L = dq::packed_layout(N, K, formats);
+    if (packed_bytes < L.total) return DQ_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint8_t *base = reinterpret_cast<uint8_t *>(packed_dev);
+    dq::PackedHeader *hdr = reinterpret_cast<dq::PackedHeader *>(base);
+    if (cudaMemsetAsync(base, 0, dq::kHeaderBytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_pack_header(hdr, cb, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_set_scale(hdr, global_scale, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (K % dq::kLutSlice != 0 && cudaMemsetAsync(base + L.lut2_off, 0, L.lut2_bytes, s) != cudaSuccess) return DQ_ERR_CUDA;
+    if (dq::launch_import_lut(2, reinterpret_cast<const uint32_t *>(lut2_planes_dev),
+                              reinterpret_cast<const uint8_t *>(lut2_scales_dev), N, K, base + L.lut2_off, s) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    if (dq::launch_pack_done(s) != cudaSuccess) return DQ_ERR_CUDA;
+    dq_weights *w = new (std::nothrow) dq_weights;
+    if (!w) return DQ_ERR_INTERNAL;
+    w->magic = kMagic;
+    cudaGetDevice(&w->device);
+    w->N = N;
+    w->K = K;
+    w->formats = formats;
+    w->base = base;
+    w->layout = L;
+    *out_host = w;
+    return DQ_OK;
+}
+
 int dq_free_weights(dq_weights *w)
 {
     if (!valid_handle(w)) return DQ_ERR_INVALID_ARG;

@@ -506,6 +506,28 @@ def test_decode_lut2_sparse_activations_and_wrong_handle(dq, oracle):
         dq.decode_linear_lut2(w3, P.to(DEV)[:1])
 
 
+@pytest.mark.parametrize("N,K,seed", [(144, 384, 31), (784, 1152, 32)])
+def test_import_canonical_lut2_round_trip(dq, oracle, N, K, seed):
+    """A LUT2 handle built from the oracle's canonical planes and scales exports the same bits again and decodes
+    like the handle packed from the master weights (K not a multiple of the 1024-weight slice: padded atoms)."""
+    W, s, planes, scales = _lut2_layer(oracle, N, K, seed)
+    w_imp = dq.import_canonical_lut2(N, K, s, torch.from_numpy(planes.view(np.int32)).to(DEV).contiguous(),
+                                     torch.from_numpy(scales).to(DEV).contiguous())
+    p2, s2, g2 = dq.export_canonical(w_imp, dq.FMT_LUT2)
+    assert np.float32(g2.cpu().numpy()[0]) == np.float32(s)
+    assert np.array_equal(p2.cpu().numpy().view(np.uint32), planes) and np.array_equal(s2.cpu().numpy(), scales)
+    w_pack = dq.pack_weights(W.to(DEV), formats=dq.FMT_LUT2)
+    X = dq_inputs.gaussian_bf16(5, K, 1.0, seed + 700).to(DEV)
+    assert torch.equal(dq.decode_linear_lut2(w_imp, X), dq.decode_linear_lut2(w_pack, X))
+    Yr, S = oracle.decode_linear_lut2(dq_inputs.bf16_to_f32_numpy(X.cpu()), planes, scales, s)
+    check_outputs(_f64(dq.decode_linear_lut2(w_imp, X)), Yr, S, "decode on an imported LUT2 handle")
+    _status_ok(dq)
+    with pytest.raises(dq.DQError):
+        dq.decode_linear(w_imp, X)                                # LUT2 only
+    rc = dq.lib().dq_import_canonical_lut2(N, K, None, None, 1.0, None, 0, None, None)
+    assert rc == 1
+
+
 def test_decode_one_hot_and_strided(dq, oracle):
     N, K = 256, 512
     W, ref = _layer(oracle, N, K, 64)
