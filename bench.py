@@ -37,9 +37,9 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the kernel named in the
 # roofline object of the same line.  None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {
-    ("gemm", "c3_gate_up27b"): 79.2e6 + 240.4e6,      # gemm_nvfp4_pair_kernel, full size
-    ("gemv", "c3_gate_up27b"): 39.04e6,               # gemv_lut_kernel<3, 384, 2>, full size, batch 1 (reads; writes are 35 KB)
-    ("gemv_nvfp4", "c3_gate_up27b"): 50.2e6,          # gemv_nvfp4_mma_kernel, small case scaled by N x K
+    ("gemm", "c3_gate_up27b"): 80.95e6 + 239.5e6,     # gemm_nvfp4_pair_kernel, full size (one-pass launch list)
+    ("gemv", "c3_gate_up27b"): 39.04e6,               # gemv_lut_kernel<3, 640, 1, 1, true>, full size, batch 1 (reads; writes are 35 KB)
+    ("gemv_nvfp4", "c3_gate_up27b"): 50.19e6,         # gemv_nvfp4_mma_kernel<640, 3>, full size (one-pass launch list)
 }
 NOMINAL_FP4_TFLOPS = 9000.0                            # dense FP4, 4 x the 2250 TFLOP/s bf16 figure
 NOMINAL_HBM_GBS = 8000.0
