@@ -153,7 +153,7 @@ def _e4m3_values(b: np.ndarray) -> np.ndarray:
     return np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7))
 
 
-@pytest.mark.parametrize("M,H,F", [(320, 512, 1024), (100, 256, 128), (700, 1024, 2304)])
+@pytest.mark.parametrize("M,H,F", [(320, 512, 1024), (100, 256, 128), (700, 1024, 2304), (1, 256, 256), (129, 384, 256)])
 def test_gate_up_gemm_with_gated_epilogue(dq, oracle, M, H, F):
     """Gate/up GEMM whose epilogue gates and quantises for the down projection (App. C.1): (a) for M > 128 the same bits
     as the GEMM followed by the fused SiLU*up quantiser; (b) against the oracle end to end -- quantised input, fp64
